@@ -1,0 +1,113 @@
+/*
+ * libenec -- ENEC lossless codec for bf16/fp16 model weights on NVIDIA B200 (sm_100a).
+ *
+ * Block-based fixed-length coding: every 16-bit value is split into its exponent field and its
+ * sign/mantissa bits (Sec. 4.2, Algorithm 1 "Split"); exponents go through the branch-free integer
+ * transform y = (b - x) mod 2^n (Sec. 5.3, Eq. 2); each group of L = 16 transformed exponents is stored
+ * with m bits per element, or with n bits when its OR needs more than m (Sec. 5.2); bits are packed with
+ * hierarchical halving bit-packing (Algorithm 2); a prefix sum over the per-block counts of wide groups
+ * gives every block's offset in the variable-length part of the stream (Sec. 5.1, Sec. 5.4); (b, n, m) are
+ * chosen per tensor from the exponent histogram (Sec. 5.5, Eq. 1, 3, 4).
+ *
+ * All pointers named d_* are DEVICE pointers, 16-byte aligned, owned by the caller. Every call only
+ * enqueues work on `stream` and returns; nothing synchronises with the host. Errors the host can see
+ * (null or misaligned pointers, unknown dtype, count >= 2^36, capacity below enec_max_compressed_size)
+ * are returned at once. Errors only the device can see (damaged stream, parameters that are not
+ * lossless, a wait that ran out) are written to *d_status if d_status is not NULL: the first error wins,
+ * the value is one of enec_status, and it stays 0 when the call succeeded. The caller zeroes *d_status.
+ * A kernel that finds an error stops touching the output; it never reads or writes out of range.
+ *
+ * The library keeps one small device scratch area per (device, stream) for the compressor (histogram
+ * and control words); it is allocated on the first compress call on that stream and kept until exit.
+ */
+#ifndef ENEC_H
+#define ENEC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { ENEC_BF16 = 0, ENEC_FP16 = 1 } enec_dtype;
+
+typedef enum {
+    ENEC_OK = 0,
+    ENEC_ERR_INVALID_ARG = -1,
+    ENEC_ERR_UNSUPPORTED_DTYPE = -2,
+    ENEC_ERR_BUFFER_TOO_SMALL = -3,
+    ENEC_ERR_BAD_STREAM = -4,
+    ENEC_ERR_PARAMS_NOT_LOSSLESS = -5,
+    ENEC_ERR_TIMEOUT = -6,
+    ENEC_ERR_CUDA = -7
+} enec_status;
+
+/* Same type as cudaStream_t; spelled out so that this header needs no CUDA header. */
+typedef struct CUstream_st* enec_stream_t;
+
+/*
+ * Upper bound, in bytes, of the stream enec_compress writes for `count` elements of `dt`: the stream
+ * layout (64-byte header, per-block prefix table, group mask, low plane, fp16 sign/mantissa-high plane,
+ * sign/mantissa byte plane, wide-group records; every section padded to 16 bytes) with n = exponent
+ * width, every group wide, maximised over m. Pure host function. Returns 0 for an unknown dtype or
+ * count >= 2^36.
+ */
+size_t enec_max_compressed_size(enec_dtype dt, size_t count);
+
+/*
+ * Compress `count` 16-bit values at d_in into d_out (Sec. 5.1 compression flow: split, histogram and
+ * parameter choice of Sec. 5.5, transform of Sec. 5.3, group widths of Sec. 5.2, Algorithm 2 packing,
+ * block-offset prefix sum). out_capacity must be at least enec_max_compressed_size(dt, count).
+ * d_out_size (device, 8-byte aligned, may be NULL) receives the stream length, which is also in the
+ * stream header. count == 0 is valid and gives a header-plus-table stream of 80 bytes.
+ */
+enec_status enec_compress(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                          size_t* d_out_size, int* d_status, enec_stream_t stream);
+
+/*
+ * As enec_compress, with the caller's (b, n, m) instead of the search of Sec. 5.5 (the paper's offline
+ * tuned mode, Sec. 6.1 "Compression Configurations"). 0 <= b < 2^E, 1 <= m <= n <= E (E = 8 for bf16,
+ * 5 for fp16). If some exponent of the tensor does not survive (b, n) the device reports
+ * ENEC_ERR_PARAMS_NOT_LOSSLESS in *d_status and writes no stream.
+ */
+enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t count, int b, int n, int m,
+                                      void* d_out, size_t out_capacity, size_t* d_out_size, int* d_status,
+                                      enec_stream_t stream);
+
+/*
+ * Decompress the stream at d_in (in_size bytes) into `count` 16-bit values at d_out (Sec. 5.1
+ * decompression flow: mask -> prefix sums -> unpack low and high parts -> inverse transform -> rejoin
+ * with sign/mantissa). dt and count must match the stream header, else ENEC_ERR_BAD_STREAM is reported in
+ * *d_status. The result is bit-identical to the tensor that was compressed.
+ */
+enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
+                            int* d_status, enec_stream_t stream);
+
+/* One tensor of a batch. All pointers are device pointers. */
+typedef struct {
+    const void* d_in;    /* decompress: stream; compress: raw values            */
+    void* d_out;         /* decompress: raw values; compress: stream            */
+    size_t count;        /* elements                                            */
+    size_t size;         /* decompress: stream bytes; compress: output capacity */
+} enec_batch_item;
+
+/*
+ * Decompress n_items streams of one dtype with a single launch (one entry per tensor, in HOST memory;
+ * the call copies the descriptors to the device on `stream`). Meant for checkpoints made of many small
+ * tensors, where one launch per tensor would be launch-bound. Same per-tensor semantics as
+ * enec_decompress; *d_status holds the first error of any tensor.
+ */
+enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, int* d_status,
+                                    enec_stream_t stream);
+
+/* Number of kernels the library has launched in this process (all entry points, all streams). */
+uint64_t enec_launch_count(void);
+
+/* Library version: 10000 * major + 100 * minor + patch. */
+int enec_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ENEC_H */

@@ -1,0 +1,133 @@
+"""GPU parity: enec_decompress (through the C-ABI) on streams written by the CPU oracle must reproduce the
+original tensor bit for bit (tolerance 0)."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import status_tensor, tensor_of, to_dev_bytes, words_of
+
+pytestmark = pytest.mark.gpu
+
+DT = {0: torch.bfloat16, 1: torch.float16}
+
+
+def gpu_decompress(stream_np, dt, count):
+    import paper_2604_03298_b200 as enec
+    d_in = to_dev_bytes(stream_np)
+    out = torch.empty(count, dtype=DT[dt], device="cuda")
+    # canary padding behind the output to catch out-of-range stores
+    guard = torch.full((count + 64,), 0x5A5A, dtype=torch.int16, device="cuda")
+    out = guard[:count].view(DT[dt])
+    status = status_tensor()
+    st = enec.enec_decompress(d_in, d_in.numel(), dt, count, out, status)
+    torch.cuda.synchronize()
+    assert (guard[count:] == 0x5A5A).all()
+    return st, int(status.item()), out
+
+
+def check_roundtrip(oracle, words, dt, params=None):
+    stream = oracle.compress(words, dt, params)
+    st, dev, out = gpu_decompress(stream, dt, words.size)
+    assert (st, dev) == (0, 0)
+    got = words_of(out)
+    if not np.array_equal(got, words):
+        bad = np.flatnonzero(got != words)
+        raise AssertionError(f"{bad.size} mismatches, first at {bad[:8]}, got {got[bad[:4]]}, want {words[bad[:4]]}")
+
+
+@pytest.mark.parametrize("dt", [0, 1])
+@pytest.mark.parametrize("count", [0, 1, 7, 16, 17, 40, 64, 100, 128, 1000, 2048, 4096, 16383, 16384, 16385,
+                                   16384 * 3 + 16, 16384 * 5 + 8191, 16384 * 37 + 129])
+def test_sizes_and_tails(oracle, dt, count):
+    g = torch.Generator().manual_seed(count + dt)
+    w = (torch.randn(count, generator=g) * 0.02).to(DT[dt]).view(torch.int16).numpy().view(np.uint16)
+    check_roundtrip(oracle, w, dt)
+
+
+@pytest.mark.parametrize("n,m", [(n, m) for n in range(1, 9) for m in range(1, n + 1)])
+def test_every_width_pair_bf16(oracle, n, m):
+    rng = np.random.default_rng(100 * n + m)
+    count = 16384 * 4 + 2048 + 40
+    half = 1 << (n - 1)
+    if n < 8:
+        x = rng.integers(max(0, 120 - (half - 1)), min(255, 120 + half) + 1, count)
+        x = np.where(rng.random(count) < 0.8, 120 - rng.integers(0, min(1 << max(m - 1, 0), half), count), x)
+    else:
+        x = rng.integers(0, 256, count)
+        x = np.where(rng.random(count) < 0.8, 120 - rng.integers(0, 1 << (m - 1), count), x)
+    words = ((x.astype(np.uint16) << 7) | rng.integers(0, 128, count).astype(np.uint16)
+             | (rng.integers(0, 2, count).astype(np.uint16) << 15)).astype(np.uint16)
+    check_roundtrip(oracle, words, 0, (120, n, m))
+
+
+@pytest.mark.parametrize("n,m", [(n, m) for n in range(1, 6) for m in range(1, n + 1)])
+def test_every_width_pair_fp16(oracle, n, m):
+    rng = np.random.default_rng(200 * n + m)
+    count = 16384 * 3 + 512 + 24
+    half = 1 << (n - 1)
+    if n < 5:
+        x = rng.integers(max(0, 12 - (half - 1)), min(31, 12 + half) + 1, count)
+    else:
+        x = rng.integers(0, 32, count)
+    x = np.where(rng.random(count) < 0.7, 12 - rng.integers(0, min(1 << (m - 1), half), count), x)
+    words = ((x.astype(np.uint16) << 10) | rng.integers(0, 1024, count).astype(np.uint16)
+             | (rng.integers(0, 2, count).astype(np.uint16) << 15)).astype(np.uint16)
+    check_roundtrip(oracle, words, 1, (12, n, m))
+
+
+@pytest.mark.parametrize("dt", [0, 1])
+def test_all_bit_patterns(oracle, dt):
+    allw = np.arange(1 << 16, dtype=np.uint16)
+    rng = np.random.default_rng(5)
+    check_roundtrip(oracle, allw, dt)
+    check_roundtrip(oracle, rng.permutation(allw), dt)
+    check_roundtrip(oracle, np.repeat(allw, 16)[:20 * 16384 + 77], dt)
+
+
+def test_mask_extremes(oracle):
+    # no group wide, every group wide, only first / only last group of a block wide
+    count = 16384 * 3
+    base = np.full(count, 123 << 7, np.uint16)
+    check_roundtrip(oracle, base, 0, (123, 6, 3))
+    allwide = base.copy()
+    allwide[::16] = 125 << 7
+    check_roundtrip(oracle, allwide, 0, (123, 6, 3))
+    first = base.copy(); first[16384] = 100 << 7
+    check_roundtrip(oracle, first, 0, (123, 6, 3))
+    last = base.copy(); last[2 * 16384 - 1] = 126 << 7
+    check_roundtrip(oracle, last, 0, (123, 6, 3))
+
+
+def test_config1_gaussian(oracle):
+    from paper_2604_03298_b200 import synth
+    spec = synth.config_specs(1)[0]
+    t = synth.make_tensor(spec, "cuda")
+    check_roundtrip(oracle, words_of(t), 0)
+
+
+def test_damaged_stream_reports_status(oracle):
+    rng = np.random.default_rng(9)
+    words = rng.integers(0x3A00, 0x3FFF, 50000).astype(np.uint16)
+    s = oracle.compress(words, 0)
+    for off, val in ((0, 0x58), (6, 1), (8, 1), (21, 0), (22, 9), (24, 77), (40, 3)):
+        bad = s.copy(); bad[off] = val
+        st, dev, _ = gpu_decompress(bad, 0, words.size)
+        assert st == 0 and dev == -4, (off, st, dev)
+    # table entry beyond the record count
+    bad = s.copy(); bad[64 + 4:64 + 8] = 0xFF
+    st, dev, _ = gpu_decompress(bad, 0, words.size)
+    assert dev == -4
+    st, dev, _ = gpu_decompress(s, 1, words.size)
+    assert dev == -4
+    st, dev, _ = gpu_decompress(s[:-16], 0, words.size)
+    assert dev == -4
+
+
+def test_host_argument_checks():
+    import paper_2604_03298_b200 as enec
+    buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(64, dtype=torch.bfloat16, device="cuda")
+    assert enec.enec_decompress(buf, 4096, 7, 64, out) == -2
+    assert enec.enec_decompress(buf[1:], 4000, 0, 64, out) == -1
+    assert enec.enec_decompress(buf, 10, 0, 64, out) == -4
+    assert enec.enec_decompress(None, 4096, 0, 64, out) == -1
