@@ -15,8 +15,42 @@ namespace enec {
 constexpr int kConsumerWarps = 8;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxStages = 4;
-constexpr uint32_t kDecodeSmemBytes = 74 * 1024;  // three CTAs per SM
+constexpr uint32_t kDecodeSmemBytes = 75 * 1024;  // three CTAs per SM
 constexpr uint32_t kStageMetaBytes = 16;
+constexpr uint32_t kNotWide = 0xFFFFu;            // rank-array entry of a group stored with m bits
+
+// Shared-memory accesses by 32-bit shared address (keeps address arithmetic in 32 bits).
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t a) {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds8(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
 
 // ---------------------------------------------------------------------------------------------------
 // Inverse of Algorithm 2 on packed bytes.
@@ -52,17 +86,17 @@ __device__ __forceinline__ uint32_t extract_bits(uint32_t v, uint32_t r, int s, 
 
 // Normalised bytes nb[i0 .. i0+7] (i0 a multiple of 8) of a plane in shared memory whose final fold has
 // half-length thalf (a multiple of 8): nb[i] sits at byte 2i (i < thalf) or 2(i - thalf) + 1.
-__device__ __forceinline__ uint2 load_octet(const uint8_t* S, uint32_t i0, uint32_t thalf) {
+__device__ __forceinline__ uint2 load_octet(uint32_t S, uint32_t i0, uint32_t thalf) {
     const bool odd = i0 >= thalf;
     const uint32_t pos = 2 * (odd ? i0 - thalf : i0);
-    const uint4 v = *reinterpret_cast<const uint4*>(S + pos);
+    const uint4 v = lds128(S + pos);
     const uint32_t sel = odd ? 0x7531u : 0x6420u;
     return make_uint2(prmt(v.x, v.y, sel), prmt(v.z, v.w, sel));
 }
 
 // out[e] (e < 2^LOG_UNITS) = packed W_IN-bit values of the eight elements j + e * n8 + (0..7) of this level.
 template <int W_IN, int LOG_UNITS>
-__device__ __forceinline__ void unpack_plane_level(const uint8_t* S, uint32_t nb_off, uint32_t j, uint32_t n8,
+__device__ __forceinline__ void unpack_plane_level(uint32_t S, uint32_t nb_off, uint32_t j, uint32_t n8,
                                                    uint32_t thalf, uint2 (&out)[1 << LOG_UNITS]) {
     constexpr int F = folds_for(W_IN);
     static_assert(F <= LOG_UNITS, "lane runs must stay whole");
@@ -89,13 +123,14 @@ __device__ __forceinline__ void unpack_plane_level(const uint8_t* S, uint32_t nb
 
 // Eight runs of eight A-bit values: y[c] = elements j + c * N/8 + (0..7) of a plane of N elements.
 template <int A>
-__device__ __forceinline__ void unpack_plane(const uint8_t* S, uint32_t j, uint32_t N, uint2 (&y)[8]) {
+__device__ __forceinline__ void unpack_plane(uint32_t S, uint32_t j, uint32_t N, uint2 (&y)[8]) {
     unpack_plane_level<A, 3>(S, 0, j, N >> 3, (N * A) >> 4, y);
 }
 
 // One element of a plane of N >= 16 elements of `a` bits, bit by bit (used only for blocks shorter than
 // 128 elements, where lane runs of eight do not exist).
-__device__ inline uint32_t unpack_plane_scalar(const uint8_t* S, uint32_t N, int a, uint32_t e) {
+template <class LoadByte>
+__device__ inline uint32_t unpack_scalar(LoadByte load_byte, uint32_t N, int a, uint32_t e) {
     const uint32_t thalf = (N * uint32_t(a)) >> 4;
     uint32_t value = 0;
     for (int q = 0; q < a; ++q) {
@@ -115,7 +150,7 @@ __device__ inline uint32_t unpack_plane_scalar(const uint8_t* S, uint32_t N, int
         }
         const uint32_t i = off + idx;
         const uint32_t pos = i < thalf ? 2 * i : 2 * (i - thalf) + 1;
-        value |= ((uint32_t(S[pos]) >> p) & 1u) << q;
+        value |= ((load_byte(pos) >> p) & 1u) << q;
     }
     return value;
 }
@@ -155,17 +190,16 @@ __device__ __forceinline__ void unpack_record_level(const uint32_t (&q)[H], int 
     }
 }
 
-// The eight H-bit values of half `half` (elements 8 half .. 8 half + 7) of the record at rp (2-byte aligned).
-template <int H>
-__device__ __forceinline__ uint2 unpack_record_half(const uint8_t* rp, uint32_t half) {
+// The sixteen H-bit values of a record, one per byte, element order.
+template <int H, class LoadWord>
+__device__ __forceinline__ uint4 unpack_record(LoadWord load_word) {
     uint32_t q[H];
 #pragma unroll
-    for (int i = 0; i < H; ++i) q[i] = *reinterpret_cast<const uint16_t*>(rp + 2 * i);
+    for (int i = 0; i < H; ++i) q[i] = load_word(i);  // 16-bit word i of the record
     uint32_t pr[8];  // pr[e] = elements 2e, 2e + 1
     unpack_record_level<H, H, 3>(q, 0, pr);
-    const uint2 h0 = make_uint2(prmt(pr[0], pr[1], 0x5410u), prmt(pr[2], pr[3], 0x5410u));
-    const uint2 h1 = make_uint2(prmt(pr[4], pr[5], 0x5410u), prmt(pr[6], pr[7], 0x5410u));
-    return half ? h1 : h0;
+    return make_uint4(prmt(pr[0], pr[1], 0x5410u), prmt(pr[2], pr[3], 0x5410u), prmt(pr[4], pr[5], 0x5410u),
+                      prmt(pr[6], pr[7], 0x5410u));
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -189,8 +223,8 @@ struct JobCtx {
 // Reads and validates the header. Returns 0 or an enec_status.
 template <int DT>
 __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
-    const Header h = *reinterpret_cast<const Header*>(job.in);
     if (job.in_size < kHeaderBytes + 16) return ENEC_ERR_BAD_STREAM;
+    const Header h = *reinterpret_cast<const Header*>(job.in);
     if (h.magic != kMagic || h.version != kVersion || h.dtype != DT || h.count != job.count ||
         h.block != kBlockElems || h.L != kGroupElems)
         return ENEC_ERR_BAD_STREAM;
@@ -214,24 +248,43 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
 }
 
 // Shared-memory layout of one pipeline stage (offsets from the stage base; all multiples of 16).
+//   meta | mask | rank array | low plane | fp16 sm-hi plane | sm bytes | raw records | expanded records
+// rank array: one u16 per group = rank of the group's record inside the block, or kNotWide.
+// expanded records: sixteen bytes per wide group (its high bits, one element per byte), rank order.
+// cap = records per block that fit; records beyond it are read from global memory by the consumers.
 struct StageLayout {
-    uint32_t meta, mask, low, smhi, sm, high, bytes;
+    uint32_t mask, rank, low, smhi, sm, raw, expanded, cap, bytes;
 };
-__device__ __forceinline__ StageLayout make_stage_layout(int dt, int m, int hbits) {
+__device__ __forceinline__ StageLayout make_stage_layout(int dt, int m, int hbits, uint32_t budget, int& nstages) {
     StageLayout L;
-    L.meta = 0;
     L.mask = kStageMetaBytes;
-    L.low = L.mask + kGroupsPerBlock / 8;
+    L.rank = L.mask + kGroupsPerBlock / 8;
+    L.low = L.rank + kGroupsPerBlock * 2;
     L.smhi = L.low + kBlockElems * uint32_t(m) / 8;
     L.sm = L.smhi + (dt == ENEC_FP16 ? kBlockElems * 3 / 8 : 0);
-    L.high = L.sm + kBlockElems;
-    L.bytes = L.high + uint32_t(align16(uint64_t(kGroupsPerBlock) * 2 * hbits + 32));  // window may start/end off-boundary
+    L.raw = L.sm + kBlockElems;
+    nstages = 2;
+    uint32_t per_stage = (budget / 2) & ~15u;
+    if (per_stage < L.raw + 48) { nstages = 1; per_stage = budget & ~15u; }
+    if (per_stage < L.raw + 48) { nstages = 0; per_stage = L.raw + 48; }
+    uint32_t cap = hbits > 0 ? (per_stage - L.raw - 48) / uint32_t(2 * hbits + 16) : 0;
+    if (cap > kGroupsPerBlock) cap = kGroupsPerBlock;
+    L.cap = cap;
+    L.expanded = L.raw + uint32_t(align16(uint64_t(cap) * 2 * hbits + 32));
+    L.bytes = L.expanded + cap * 16;
+    if (nstages == 2) {
+        int more = int(budget / L.bytes);
+        nstages = more > kMaxStages ? kMaxStages : more;
+    }
     return L;
 }
 
 struct RunCtx {
-    const uint8_t* sm;    // shared: sign/mantissa bytes of the block
-    const uint8_t* high;  // shared: first record of the block
+    uint32_t sm;          // shared address: sign/mantissa bytes of the block
+    uint32_t rank;        // shared address: rank array
+    uint32_t expanded;    // shared address: expanded records
+    uint32_t cap;         // records expanded in shared memory
+    const uint8_t* high;  // global: first record of the block
     uint16_t* out;        // global: first element of the block
     uint32_t real;        // real elements in the block
     uint32_t c4_or_h, fix, s4, b4;  // packed transform constants
@@ -256,23 +309,30 @@ __device__ __forceinline__ uint32_t inverse_transform4(const RunCtx& r, uint32_t
     return x;
 }
 
-// Finishes eight consecutive elements e0 .. e0+7 of a block: wide-group high bits, inverse transform,
+// High bits of eight elements of a wide group whose record was not expanded in shared memory.
+template <int HB>
+__device__ __noinline__ uint2 record_half_from_global(const uint8_t* rp, uint32_t second_half) {
+    const uint4 v = unpack_record<HB>([&](int i) { return uint32_t(*reinterpret_cast<const uint16_t*>(rp + 2 * i)); });
+    return second_half ? make_uint2(v.z, v.w) : make_uint2(v.x, v.y);
+}
+
+// Finishes eight consecutive elements e0 .. e0+7 of a block: high bits of wide groups, inverse transform,
 // rejoin with sign/mantissa, store.
 template <int DT, int M, int HB>
-__device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, uint32_t e0, uint32_t mword,
-                                           uint32_t mprefix, bool active) {
+__device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, uint32_t e0, bool active) {
     if constexpr (HB > 0) {
-        const uint32_t bit = (e0 >> 4) & 31;
-        if ((mword >> bit) & 1) {
-            const uint32_t rank = mprefix + __popc(mword & ((1u << bit) - 1));
-            const uint2 hi = unpack_record_half<HB>(r.high + rank * (2 * HB), (e0 >> 3) & 1);
+        const uint32_t rk = lds16(r.rank + ((e0 >> 4) << 1));
+        if (rk != kNotWide) {
+            uint2 hi;
+            if (rk < r.cap) hi = lds64(r.expanded + rk * 16 + (e0 & 8));
+            else hi = record_half_from_global<HB>(r.high + rk * (2 * HB), e0 & 8);
             y.x |= hi.x << M;
             y.y |= hi.y << M;
         }
     }
     const uint32_t x0 = inverse_transform4<DT>(r, y.x);
     const uint32_t x1 = inverse_transform4<DT>(r, y.y);
-    const uint2 smv = *reinterpret_cast<const uint2*>(r.sm + e0);
+    const uint2 smv = lds64(r.sm + e0);
     uint32_t lo0, lo1, hi0, hi1;
     if (DT == ENEC_BF16) {
         // word = sign << 15 | x << 7 | mant7 ; sm byte = sign << 7 | mant7
@@ -296,32 +356,17 @@ __device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, u
     if (e0 + 8 <= r.real) {
         *reinterpret_cast<uint4*>(r.out + e0) = w;
     } else if (e0 < r.real) {
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-        for (uint32_t i = 0; e0 + i < r.real; ++i) r.out[e0 + i] = uint16_t(ww[i >> 1] >> (16 * (i & 1)));
+        for (uint32_t i = 0; e0 + i < r.real; ++i) {
+            const uint32_t pair = (i >> 1) == 0 ? w.x : (i >> 1) == 1 ? w.y : (i >> 1) == 2 ? w.z : w.w;
+            r.out[e0 + i] = uint16_t(pair >> (16 * (i & 1)));
+        }
     }
 }
 
 // One block, all consumer threads. tid = 0..255. N = padded block length.
 template <int DT, int M, int HB>
-__device__ __forceinline__ void decode_block(const RunCtx& r, const uint8_t* s_low, const uint8_t* s_smhi,
-                                             const uint32_t* s_mask, uint32_t N, uint32_t tid) {
-    const uint32_t lane = tid & 31;
-    const uint32_t groups = N >> 4;
-    // per-warp exclusive popcount prefix over the block's mask words
-    uint32_t mw = 0;
-    if (lane * 32 < groups) {
-        mw = s_mask[lane];
-        if (groups - lane * 32 < 32) mw &= (1u << (groups - lane * 32)) - 1;
-    }
-    if (HB == 0) mw = 0;
-    uint32_t incl = __popc(mw);
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-        if (lane >= uint32_t(d)) incl += t;
-    }
-    const uint32_t excl = incl - __popc(mw);
-
+__device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, uint32_t s_smhi, uint32_t N,
+                                             uint32_t tid) {
     if (N >= 128) {
         const uint32_t items = N >> 6;
         const uint32_t n8 = N >> 3;
@@ -334,34 +379,67 @@ __device__ __forceinline__ void decode_block(const RunCtx& r, const uint8_t* s_l
             unpack_plane<M>(s_low, j, N, y);
             if (DT == ENEC_FP16) unpack_plane<3>(s_smhi, j, N, hs);
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t e0 = c * n8 + j;
-                const uint32_t wi = e0 >> 9;
-                const uint32_t mword = __shfl_sync(0xFFFFFFFFu, mw, wi);
-                const uint32_t mpre = __shfl_sync(0xFFFFFFFFu, excl, wi);
-                finish_run<DT, M, HB>(r, y[c], DT == ENEC_FP16 ? hs[c] : make_uint2(0, 0), e0, mword, mpre, active);
-            }
+            for (int c = 0; c < 8; ++c)
+                finish_run<DT, M, HB>(r, y[c], DT == ENEC_FP16 ? hs[c] : make_uint2(0, 0), c * n8 + j, active);
         }
-    } else if (tid < 32) {
-        // short tail block (16, 32 or 64 elements): one run of eight per lane, values rebuilt bit by bit
-        const bool active = lane * 8 < N;
-        const uint32_t e0 = active ? lane * 8 : 0;
+    } else {
+        // short tail block (16, 32 or 64 elements): one run of eight per thread, values rebuilt bit by bit
+        if (tid * 8 >= N) return;
+        const uint32_t e0 = tid * 8;
         uint32_t yb[2] = {0, 0}, hb[2] = {0, 0};
         for (uint32_t i = 0; i < 8; ++i) {
-            yb[i >> 2] |= unpack_plane_scalar(s_low, N, M, e0 + i) << (8 * (i & 3));
-            if (DT == ENEC_FP16) hb[i >> 2] |= unpack_plane_scalar(s_smhi, N, 3, e0 + i) << (8 * (i & 3));
+            yb[i >> 2] |= unpack_scalar([&](uint32_t p) { return lds8(s_low + p); }, N, M, e0 + i) << (8 * (i & 3));
+            if (DT == ENEC_FP16)
+                hb[i >> 2] |= unpack_scalar([&](uint32_t p) { return lds8(s_smhi + p); }, N, 3, e0 + i) << (8 * (i & 3));
         }
-        const uint32_t mword = __shfl_sync(0xFFFFFFFFu, mw, 0);
-        const uint32_t mpre = __shfl_sync(0xFFFFFFFFu, excl, 0);
-        finish_run<DT, M, HB>(r, make_uint2(yb[0], yb[1]), make_uint2(hb[0], hb[1]), e0, mword, mpre, active);
+        finish_run<DT, M, HB>(r, make_uint2(yb[0], yb[1]), make_uint2(hb[0], hb[1]), e0, true);
     }
 }
 
+// Loader/expander warp, one block: per-group ranks from the mask, then the block's first `cap` records
+// expanded to sixteen bytes each. All 32 lanes.
+template <int HB>
+__device__ __forceinline__ void expand_records(uint32_t s_raw, uint32_t s_expanded, uint32_t count, uint32_t lane) {
+    for (uint32_t i = lane; i < count; i += 32) {
+        const uint32_t rp = s_raw + i * (2 * HB);
+        const uint4 v = unpack_record<HB>([&](int w) { return lds16(rp + 2 * w); });
+        sts128(s_expanded + i * 16, v);
+    }
+}
+
+__device__ __forceinline__ uint32_t build_rank_array(uint32_t s_mask, uint32_t s_rank, uint32_t N, uint32_t lane) {
+    const uint32_t groups = N >> 4;
+    uint32_t mw = 0;
+    if (lane * 32 < groups) {
+        mw = lds32(s_mask + 4 * lane);
+        if (groups - lane * 32 < 32) mw &= (1u << (groups - lane * 32)) - 1;
+    }
+    uint32_t incl = __popc(mw);
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= uint32_t(d)) incl += t;
+    }
+    uint32_t run = incl - __popc(mw);
+    if (lane * 32 < groups) {
+#pragma unroll
+        for (int b = 0; b < 32; b += 2) {
+            const uint32_t r0 = (mw >> b) & 1 ? run : kNotWide;
+            run += (mw >> b) & 1;
+            const uint32_t r1 = (mw >> (b + 1)) & 1 ? run : kNotWide;
+            run += (mw >> (b + 1)) & 1;
+            sts32(s_rank + (lane * 32 + b) * 2, r0 | (r1 << 16));
+        }
+    }
+    return __shfl_sync(0xFFFFFFFFu, incl, 31);  // wide groups in the block according to the mask
+}
+
 struct DecodeShared {
-    uint64_t full[kMaxStages];
-    uint64_t empty[kMaxStages];
+    uint64_t full[kMaxStages];   // bulk copies of a stage have landed
+    uint64_t ready[kMaxStages];  // rank array and expanded records of a stage are written
+    uint64_t empty[kMaxStages];  // all consumer warps are done with a stage
     int abort;
-    int pad[15];
+    int pad[7];
 };
 static_assert(sizeof(DecodeShared) == 128, "control area is 128 bytes");
 
@@ -381,12 +459,27 @@ static_assert(sizeof(DecodeShared) == 128, "control area is 128 bytes");
     X(DT, 7, 0) X(DT, 7, 1)                                                                           \
     X(DT, 8, 0)
 
+// Bounded wait by lane 0 with the result broadcast to the warp; also gives up when the CTA aborts.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t lane) {
+    int ok = 0;
+    if (lane == 0) {
+        for (uint32_t it = 0; it < (1u << 22); ++it) {
+            if (mbar_try_wait(bar, parity)) { ok = 1; break; }
+            if (*abort_flag) break;
+            if (it > 16) __nanosleep(64);
+        }
+    }
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    if (ok && lane != 0) mbar_try_wait(bar, parity);  // acquire in every lane
+    return ok != 0;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
 enec_decode_kernel(DecodeJob job, int* status) {
     extern __shared__ __align__(128) uint8_t smem[];
     DecodeShared* ctl = reinterpret_cast<DecodeShared*>(smem);
-    uint8_t* stages = smem + sizeof(DecodeShared);
+    const uint32_t stages = smem_u32(smem) + uint32_t(sizeof(DecodeShared));
 
     JobCtx jc;
     const int err = load_job<DT>(job, jc);
@@ -395,16 +488,16 @@ enec_decode_kernel(DecodeJob job, int* status) {
         return;
     }
     const int hbits = jc.n - jc.m;
-    const StageLayout L = make_stage_layout(DT, jc.m, hbits);
-    int nstages = int((kDecodeSmemBytes - sizeof(DecodeShared)) / L.bytes);
-    if (nstages > kMaxStages) nstages = kMaxStages;
-    if (nstages < 1) {  // cannot happen for valid (m, n): the largest stage is below 54 KB
+    int nstages = 0;
+    const StageLayout L = make_stage_layout(DT, jc.m, hbits, kDecodeSmemBytes - uint32_t(sizeof(DecodeShared)), nstages);
+    if (nstages < 1) {  // cannot happen for valid (m, n): the fixed part of a stage is below 40 KB
         if (threadIdx.x == 0 && blockIdx.x == 0) report(status, ENEC_ERR_BAD_STREAM);
         return;
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < nstages; ++s) {
             mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->ready[s], 1);
             mbar_init(&ctl->empty[s], kConsumerWarps);
         }
         ctl->abort = 0;
@@ -415,56 +508,106 @@ enec_decode_kernel(DecodeJob job, int* status) {
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lane = threadIdx.x & 31;
     volatile int* abort_flag = &ctl->abort;
+    const uint32_t n_mine = jc.nblocks > blockIdx.x ? (jc.nblocks - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint32_t S = uint32_t(nstages);
 
     if (warp == kConsumerWarps) {
-        // ---------------- producer ----------------
-        if (lane != 0) return;
+        // ---------------- loader + expander warp ----------------
         const uint32_t* table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
-        uint32_t issued = 0;
-        for (uint32_t k = blockIdx.x; k < jc.nblocks; k += gridDim.x, ++issued) {
-            const int s = int(issued % uint32_t(nstages));
-            const uint32_t use = issued / uint32_t(nstages);
-            if (use > 0 && !mbar_wait_bounded(&ctl->empty[s], (use - 1) & 1)) {
-                *abort_flag = 1;
-                report(status, ENEC_ERR_TIMEOUT);
-                break;
+        uint32_t next_load = 0, next_exp = 0;
+        uint32_t t0 = 0, t1 = 0;  // table entries of block next_load (lane 0)
+        if (lane == 0 && n_mine) { t0 = table[blockIdx.x]; t1 = table[blockIdx.x + 1]; }
+        bool failed = false;
+        while (next_exp < n_mine && !failed) {
+            // issue every load that has a free stage; block only when there is nothing to expand
+            while (next_load < n_mine && next_load < next_exp + S) {
+                const uint32_t s = next_load % S, use = next_load / S;
+                if (use > 0) {
+                    bool free_now;
+                    if (next_exp < next_load) {
+                        int f = lane == 0 ? int(mbar_try_wait(&ctl->empty[s], (use - 1) & 1)) : 0;
+                        free_now = __shfl_sync(0xFFFFFFFFu, f, 0) != 0;
+                        if (!free_now) break;
+                    } else if (!warp_wait(&ctl->empty[s], (use - 1) & 1, abort_flag, lane)) {
+                        failed = true;
+                        break;
+                    }
+                }
+                int bad = 0;
+                if (lane == 0) {
+                    const uint32_t k = blockIdx.x + next_load * gridDim.x;
+                    const bool tail = (k + 1 == jc.nblocks);
+                    const uint32_t N = tail ? jc.tail_padded : kBlockElems;
+                    const uint32_t real = tail ? jc.tail_real : kBlockElems;
+                    const uint64_t h0 = jc.off_high + uint64_t(t0) * (2 * hbits);
+                    const uint64_t w0 = h0 & ~uint64_t(15);
+                    bad = t1 < t0 || t1 - t0 > (N >> 4) || t1 > jc.a_total;
+                    if (!bad) {
+                        uint32_t staged = t1 - t0 < L.cap ? t1 - t0 : L.cap;   // records staged and expanded
+                        if (hbits == 0) staged = 0;
+                        const uint64_t w1 = align16(h0 + uint64_t(staged) * (2 * hbits));
+                        const uint32_t mask_bytes = uint32_t(align16(((N >> 4) + 7) / 8));
+                        const uint32_t low_bytes = uint32_t(align16(uint64_t(N) * jc.m / 8));
+                        const uint32_t smhi_bytes = DT == ENEC_FP16 ? uint32_t(align16(uint64_t(N) * 3 / 8)) : 0;
+                        const uint32_t sm_bytes = uint32_t(align16(real));
+                        const uint32_t raw_bytes = staged ? uint32_t(w1 - w0) : 0;
+                        uint8_t* st = smem + sizeof(DecodeShared) + size_t(s) * L.bytes;
+                        uint32_t* meta = reinterpret_cast<uint32_t*>(st);
+                        meta[0] = uint32_t(h0 - w0);  // offset of the first record inside the staged window
+                        meta[1] = staged;
+                        meta[2] = t1 - t0;
+                        mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes);
+                        bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
+                        bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
+                        if (DT == ENEC_FP16)
+                            bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
+                        bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
+                        if (raw_bytes) bulk_g2s(st + L.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
+                        if (next_load + 1 < n_mine) { t0 = table[k + gridDim.x]; t1 = table[k + gridDim.x + 1]; }
+                    }
+                }
+                if (__shfl_sync(0xFFFFFFFFu, bad, 0)) {
+                    if (lane == 0) { *abort_flag = 1; report(status, ENEC_ERR_BAD_STREAM); }
+                    failed = true;
+                    break;
+                }
+                ++next_load;
             }
-            if (*abort_flag) break;
-            const bool tail = (k + 1 == jc.nblocks);
-            const uint32_t N = tail ? jc.tail_padded : kBlockElems;
-            const uint32_t real = tail ? jc.tail_real : kBlockElems;
-            const uint32_t t0 = table[k], t1 = table[k + 1];
-            uint8_t* st = stages + size_t(s) * L.bytes;
-            uint32_t* meta = reinterpret_cast<uint32_t*>(st + L.meta);
-            const uint64_t h0 = jc.off_high + uint64_t(t0) * (2 * hbits);
-            const uint64_t h1 = jc.off_high + uint64_t(t1) * (2 * hbits);
-            const uint64_t w0 = h0 & ~uint64_t(15), w1 = align16(h1);
-            bool bad = t1 < t0 || t1 - t0 > (N >> 4) || t1 > jc.a_total || w1 > jc.total;
-            if (bad) {
-                *abort_flag = 1;
-                report(status, ENEC_ERR_BAD_STREAM);
-                break;
+            if (failed || next_exp >= next_load) continue;
+            // expand the oldest loaded block
+            const uint32_t s = next_exp % S, use = next_exp / S;
+            if (!warp_wait(&ctl->full[s], use & 1, abort_flag, lane)) { failed = true; break; }
+            const uint32_t k = blockIdx.x + next_exp * gridDim.x;
+            const uint32_t N = (k + 1 == jc.nblocks) ? jc.tail_padded : kBlockElems;
+            const uint32_t st = stages + s * L.bytes;
+            const uint32_t first = lds32(st), staged = lds32(st + 4), expect = lds32(st + 8);
+            if (hbits > 0) {
+                const uint32_t wide = build_rank_array(st + L.mask, st + L.rank, N, lane);
+                if (wide != expect) {  // the prefix table must agree with the mask
+                    if (lane == 0) { *abort_flag = 1; report(status, ENEC_ERR_BAD_STREAM); }
+                    failed = true;
+                    break;
+                }
+                switch (hbits) {
+                    case 1: expand_records<1>(st + L.raw + first, st + L.expanded, staged, lane); break;
+                    case 2: expand_records<2>(st + L.raw + first, st + L.expanded, staged, lane); break;
+                    case 3: expand_records<3>(st + L.raw + first, st + L.expanded, staged, lane); break;
+                    case 4: expand_records<4>(st + L.raw + first, st + L.expanded, staged, lane); break;
+                    case 5: expand_records<5>(st + L.raw + first, st + L.expanded, staged, lane); break;
+                    case 6: expand_records<6>(st + L.raw + first, st + L.expanded, staged, lane); break;
+                    default: expand_records<7>(st + L.raw + first, st + L.expanded, staged, lane); break;
+                }
             }
-            const uint32_t mask_bytes = uint32_t(align16(((N >> 4) + 7) / 8));
-            const uint32_t low_bytes = uint32_t(align16(uint64_t(N) * jc.m / 8));
-            const uint32_t smhi_bytes = DT == ENEC_FP16 ? uint32_t(align16(uint64_t(N) * 3 / 8)) : 0;
-            const uint32_t sm_bytes = uint32_t(align16(real));
-            const uint32_t high_bytes = (hbits > 0 && t1 > t0) ? uint32_t(w1 - w0) : 0;
-            meta[0] = uint32_t(h0 - w0);  // offset of the block's first record inside the staged window
-            meta[1] = t1 - t0;
-            mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + high_bytes);
-            bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
-            bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
-            if (DT == ENEC_FP16)
-                bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
-            bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
-            if (high_bytes) bulk_g2s(st + L.high, jc.in + w0, high_bytes, &ctl->full[s]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->ready[s]);
+            ++next_exp;
         }
-        if (*abort_flag) {
-            // let copies still in flight land before the CTA's shared memory is released
-            const uint32_t first = issued > uint32_t(nstages) ? issued - uint32_t(nstages) : 0;
-            for (uint32_t i = first; i < issued; ++i)
-                mbar_wait_bounded(&ctl->full[i % uint32_t(nstages)], (i / uint32_t(nstages)) & 1);
+        if (failed) {
+            if (lane == 0) {
+                if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
+                // let copies still in flight land before the CTA's shared memory is released
+                for (uint32_t i = next_exp; i < next_load; ++i) mbar_wait_bounded(&ctl->full[i % S], (i / S) & 1);
+            }
         }
         return;
     }
@@ -479,49 +622,36 @@ enec_decode_kernel(DecodeJob job, int* status) {
         r.fix = ~rep4(c) & 0x80808080u;
         r.b4 = rep4(uint32_t(jc.b));
         r.n = jc.n;
+        r.cap = L.cap;
     }
     const int code = jc.m * 8 + hbits;
-    uint32_t done = 0;
-    for (uint32_t k = blockIdx.x; k < jc.nblocks; k += gridDim.x, ++done) {
-        const int s = int(done % uint32_t(nstages));
-        const uint32_t use = done / uint32_t(nstages);
-        bool ok = true;
-        if (lane == 0) {
-            ok = false;
-            for (uint32_t it = 0; it < (1u << 22); ++it) {
-                if (mbar_try_wait(&ctl->full[s], use & 1)) { ok = true; break; }
-                if (*abort_flag) break;
-                if (it > 32) __nanosleep(128);
-            }
-            if (!ok && !*abort_flag) {
-                *abort_flag = 1;
-                report(status, ENEC_ERR_TIMEOUT);
-            }
+    for (uint32_t i = 0; i < n_mine; ++i) {
+        const uint32_t s = i % S, use = i / S;
+        if (!warp_wait(&ctl->ready[s], use & 1, abort_flag, lane)) {
+            if (lane == 0 && !*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
+            break;
         }
-        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        if (lane != 0) mbar_try_wait(&ctl->full[s], use & 1);  // acquire the staged bytes in every lane
+        mbar_try_wait(&ctl->full[s], use & 1);  // the staged bytes themselves (already complete)
+        const uint32_t k = blockIdx.x + i * gridDim.x;
         const bool tail = (k + 1 == jc.nblocks);
         const uint32_t N = tail ? jc.tail_padded : kBlockElems;
-        const uint8_t* st = stages + size_t(s) * L.bytes;
-        const uint32_t* meta = reinterpret_cast<const uint32_t*>(st + L.meta);
+        const uint32_t st = stages + s * L.bytes;
         r.sm = st + L.sm;
-        r.high = st + L.high + meta[0];
+        r.rank = st + L.rank;
+        r.expanded = st + L.expanded;
+        r.high = jc.in + jc.off_high + uint64_t(reinterpret_cast<const uint32_t*>(jc.in + jc.off_table)[k]) * (2 * hbits);
         r.out = jc.out + uint64_t(k) * kBlockElems;
         r.real = tail ? jc.tail_real : kBlockElems;
-        const uint8_t* s_low = st + L.low;
-        const uint8_t* s_smhi = st + L.smhi;
-        const uint32_t* s_mask = reinterpret_cast<const uint32_t*>(st + L.mask);
         switch (code) {
 #define ENEC_CASE(DTV, MV, HV)                                                        \
     case MV * 8 + HV:                                                                 \
-        decode_block<DTV, MV, HV>(r, s_low, s_smhi, s_mask, N, threadIdx.x);          \
+        decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, threadIdx.x);        \
         break;
             ENEC_FOR_EACH_MH(ENEC_CASE, DT)
 #undef ENEC_CASE
 #define ENEC_CASE(DTV, MV, HV)                                                        \
     case MV * 8 + HV:                                                                 \
-        if constexpr (DTV == ENEC_BF16) decode_block<DTV, MV, HV>(r, s_low, s_smhi, s_mask, N, threadIdx.x); \
+        if constexpr (DTV == ENEC_BF16) decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, threadIdx.x); \
         break;
             ENEC_FOR_EACH_MH_BF16_ONLY(ENEC_CASE, DT)
 #undef ENEC_CASE

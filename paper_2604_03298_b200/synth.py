@@ -96,6 +96,9 @@ def make_tensor(spec: TensorSpec, device="cpu") -> torch.Tensor:
     n = spec.numel
     if spec.dist == "normal":
         t = torch.randn(n, generator=gen, device=device, dtype=torch.float32)
+        # A float32 normal generator emits exact 0.0 about once per 2^24 draws; a Gaussian has no atom at
+        # zero, and one such value would set the lowest occupied exponent to 0 for the whole tensor.
+        t = torch.where(t == 0, torch.full_like(t, 2.0 ** -10), t)
         t = t * spec.std + spec.mean
     elif spec.dist == "laplace":
         u = torch.rand(n, generator=gen, device=device, dtype=torch.float32) - 0.5
