@@ -1,8 +1,11 @@
 // C-ABI entry points of libenec (see include/enec.h). Host-side validation and kernel launches only.
 #include <atomic>
+#include <map>
 #include <mutex>
+#include <utility>
 
 #include "enec_decode.cuh"
+#include "enec_encode.cuh"
 
 namespace enec {
 
@@ -11,6 +14,7 @@ std::atomic<uint64_t> g_launches{0};
 struct DeviceInfo {
     int sms = 0;
     bool decode_attr_set[2] = {false, false};
+    bool hist_attr_set[2] = {false, false};
 };
 
 static DeviceInfo& device_info(int dev) {
@@ -43,6 +47,96 @@ static enec_status launch_decode(const DecodeJob& job, uint32_t nblocks, int* d_
     return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
 
+
+// Device scratch of the compressor, one area per (device, stream): control words and one state word per
+// block. Grown when a larger tensor arrives; outgrown areas are kept until exit because work that uses
+// them may still be queued.
+struct ScratchArea {
+    uint8_t* ptr = nullptr;
+    size_t bytes = 0;
+};
+
+static enec_status get_scratch(int dev, cudaStream_t stream, size_t need, uint8_t** out) {
+    static std::mutex mu;
+    static std::map<std::pair<int, cudaStream_t>, ScratchArea> areas;
+    std::lock_guard<std::mutex> lock(mu);
+    ScratchArea& a = areas[std::make_pair(dev, stream)];
+    if (a.bytes < need) {
+        size_t bytes = a.bytes ? a.bytes : size_t(64) << 10;
+        while (bytes < need) bytes *= 2;
+        void* p = nullptr;
+        if (cudaMalloc(&p, bytes) != cudaSuccess) return ENEC_ERR_CUDA;
+        a.ptr = static_cast<uint8_t*>(p);
+        a.bytes = bytes;
+    }
+    *out = a.ptr;
+    return ENEC_OK;
+}
+
+template <int DT>
+static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool search, int* d_status, DeviceInfo& info,
+                                 cudaStream_t stream) {
+    if (search) {
+        const uint32_t smem = HistShape<DT>::kWarpBytes * (kHistThreads / 32);
+        if (!info.hist_attr_set[DT]) {
+            if (cudaFuncSetAttribute(enec_histogram_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) !=
+                cudaSuccess)
+                return ENEC_ERR_CUDA;
+            info.hist_attr_set[DT] = true;
+        }
+        const uint64_t chunks = job.count >> 3;
+        uint64_t grid = (chunks + kHistThreads - 1) / kHistThreads;
+        if (grid > uint64_t(info.sms) * 3) grid = uint64_t(info.sms) * 3;
+        if (grid == 0) grid = 1;
+        enec_histogram_kernel<DT><<<uint32_t(grid), kHistThreads, smem, stream>>>(job.in, job.count, job.ctl);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    enec_encode_kernel<DT><<<nblocks, kEncodeThreads, 0, stream>>>(job, d_status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
+}
+
+static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count, bool with_params, int b, int n,
+                                   int m, void* d_out, size_t out_capacity, size_t* d_out_size, int* d_status,
+                                   cudaStream_t stream) {
+    if (dt != ENEC_BF16 && dt != ENEC_FP16) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if ((!d_in && count) || !d_out || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out) ||
+        (reinterpret_cast<uintptr_t>(d_out_size) & 7))
+        return ENEC_ERR_INVALID_ARG;
+    const int E = exp_bits(dt);
+    if (with_params && (n < 1 || n > E || m < 1 || m > n || b < 0 || b >= (1 << E))) return ENEC_ERR_INVALID_ARG;
+    if (out_capacity < enec_max_compressed_size(dt, count)) return ENEC_ERR_BUFFER_TOO_SMALL;
+    unsigned long long* out_size = reinterpret_cast<unsigned long long*>(d_out_size);
+    if (count == 0) {
+        // no exponent occurs: the search of Sec. 5.5 has nothing to minimise and keeps (0, 1, 1)
+        enec_encode_empty_kernel<<<1, 32, 0, stream>>>(static_cast<uint8_t*>(d_out), int(dt), with_params ? b : 0,
+                                                      with_params ? n : 1, with_params ? m : 1, out_size);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
+    DeviceInfo& info = device_info(dev);
+    const Geometry g = make_geometry(count);
+    const size_t need = kControlBytes + size_t(g.nblocks) * sizeof(unsigned long long);
+    uint8_t* scratch = nullptr;
+    const enec_status st = get_scratch(dev, stream, need, &scratch);
+    if (st != ENEC_OK) return st;
+    if (cudaMemsetAsync(scratch, 0, need, stream) != cudaSuccess) return ENEC_ERR_CUDA;
+    EncodeJob job;
+    job.in = static_cast<const uint16_t*>(d_in);
+    job.out = static_cast<uint8_t*>(d_out);
+    job.count = count;
+    job.ctl = reinterpret_cast<EncodeControl*>(scratch);
+    job.state = reinterpret_cast<unsigned long long*>(scratch + kControlBytes);
+    job.out_size = out_size;
+    job.b = b; job.n = n; job.m = m;
+    job.from_search = with_params ? 0 : 1;
+    job.check = with_params ? 1 : 0;
+    return dt == ENEC_BF16 ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream)
+                           : launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream);
+}
+
 }  // namespace enec
 
 using namespace enec;
@@ -73,13 +167,17 @@ enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, siz
                            : launch_decode<ENEC_FP16>(job, g.nblocks, d_status, stream);
 }
 
-enec_status enec_compress(const void*, enec_dtype, size_t, void*, size_t, size_t*, int*, enec_stream_t) {
-    return ENEC_ERR_CUDA;  // TEMP
+enec_status enec_compress(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                          size_t* d_out_size, int* d_status, enec_stream_t stream) {
+    return compress_common(d_in, dt, count, false, 0, 0, 0, d_out, out_capacity, d_out_size, d_status, stream);
 }
-enec_status enec_compress_with_params(const void*, enec_dtype, size_t, int, int, int, void*, size_t, size_t*, int*,
-                                      enec_stream_t) {
-    return ENEC_ERR_CUDA;  // TEMP
+
+enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t count, int b, int n, int m,
+                                      void* d_out, size_t out_capacity, size_t* d_out_size, int* d_status,
+                                      enec_stream_t stream) {
+    return compress_common(d_in, dt, count, true, b, n, m, d_out, out_capacity, d_out_size, d_status, stream);
 }
+
 enec_status enec_decompress_batched(const enec_batch_item*, int, enec_dtype, int*, enec_stream_t) {
     return ENEC_ERR_CUDA;  // TEMP
 }

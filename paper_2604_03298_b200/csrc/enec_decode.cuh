@@ -19,39 +19,6 @@ constexpr uint32_t kDecodeSmemBytes = 75 * 1024;  // three CTAs per SM
 constexpr uint32_t kStageMetaBytes = 16;
 constexpr uint32_t kNotWide = 0xFFFFu;            // rank-array entry of a group stored with m bits
 
-// Shared-memory accesses by 32-bit shared address (keeps address arithmetic in 32 bits).
-__device__ __forceinline__ uint4 lds128(uint32_t a) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ uint2 lds64(uint32_t a) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ uint32_t lds32(uint32_t a) {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ uint32_t lds16(uint32_t a) {
-    uint16_t v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ uint32_t lds8(uint32_t a) {
-    uint32_t v;
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
-}
-
 // ---------------------------------------------------------------------------------------------------
 // Inverse of Algorithm 2 on packed bytes.
 //
@@ -64,17 +31,6 @@ __device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
 // elements {j + c N/8 + i : c, i < 8} from a few 16-byte shared-memory loads with shifts and masks whose
 // amounts are compile-time constants.
 // ---------------------------------------------------------------------------------------------------
-__host__ __device__ constexpr int folds_for(int w) {
-    int f = 0;
-    while ((w << f) < 8) ++f;
-    return f;
-}
-__host__ __device__ constexpr int bitrev(int t, int f) {
-    int r = 0;
-    for (int i = 0; i < f; ++i) r |= ((t >> i) & 1) << (f - 1 - i);
-    return r;
-}
-
 // bits [s, s + w) of the 16-bit lanes (v | r << 8), four lanes per register, one lane per byte
 __device__ __forceinline__ uint32_t extract_bits(uint32_t v, uint32_t r, int s, int w) {
     const uint32_t m = (1u << w) - 1;

@@ -1,0 +1,833 @@
+// Compression kernels (Sec. 5.1 compression flow).
+//
+//   enec_histogram_kernel  Sec. 5.5 phase 1 (exponent histogram of the whole tensor) with the search of
+//                          phases 2 and 3 (Eq. 1, 3, 4) run by the last CTA to finish.
+//   enec_encode_kernel     one CTA per 16384-element block: split, transform (Eq. 2), group widths
+//                          (Sec. 5.2), Algorithm 2 on packed bytes for the low plane and for the records
+//                          of wide groups, and the block-offset prefix sum as a decoupled look-back over
+//                          per-block state words, so the input is read once.
+//   enec_encode_empty_kernel  the 80-byte stream of an empty tensor.
+//
+// Blocks are handed out by an atomic ticket, so a block's predecessors are always resident or finished
+// and every look-back wait ends; the wait is bounded all the same and ends in ENEC_ERR_TIMEOUT.
+#pragma once
+
+#include "enec_common.cuh"
+
+namespace enec {
+
+constexpr int kEncodeThreads = 256;
+constexpr int kHistThreads = 256;
+constexpr uint32_t kControlBytes = 4096;  // control area in front of the per-block state words
+
+// Device scratch of one compress call: control words, then one 64-bit state word per block.
+struct alignas(16) EncodeControl {
+    unsigned long long hist[256];  // exponent histogram (2^E bins used)
+    uint32_t ticket;               // next block to hand out
+    uint32_t hist_done;            // CTAs of the histogram kernel that have finished
+    uint32_t error;                // some block failed; the header is not written
+    int b, n, m;                   // result of the parameter search
+};
+static_assert(sizeof(EncodeControl) <= kControlBytes, "control area");
+
+// state word: bits 63..62 = kind, bits 31..0 = value
+constexpr unsigned long long kStateAggregate = 1ull << 62;  // value = wide groups in the block
+constexpr unsigned long long kStatePrefix = 2ull << 62;     // value = wide groups up to and including the block
+constexpr unsigned long long kStatePoison = 3ull << 62;     // a predecessor failed
+
+struct EncodeJob {
+    const uint16_t* in;
+    uint8_t* out;
+    uint64_t count;
+    EncodeControl* ctl;
+    unsigned long long* state;
+    unsigned long long* out_size;  // device, may be null
+    int b, n, m;                   // used when from_search == 0
+    int from_search;               // take (b, n, m) from ctl
+    int check;                     // verify that (b, n) keeps every exponent
+};
+
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Sec. 5.5 phase 1: histogram of the exponent field.
+//
+// Each lane keeps private 8-bit counters in shared memory (four bins per 32-bit word, the word's bank
+// equal to the lane), so counting needs neither atomics nor bank conflicts whatever the distribution;
+// a warp folds its counters into the CTA's 32-bit histogram every 31 loads of eight values (248 < 256).
+// ---------------------------------------------------------------------------------------------------
+template <int DT>
+struct HistShape {
+    static constexpr int E = DT == ENEC_BF16 ? 8 : 5;
+    static constexpr int kBins = 1 << E;
+    static constexpr int kQuads = kBins / 4;             // words per lane
+    static constexpr int kWarpBytes = kQuads * 128;      // counters of one warp
+};
+
+// byte address (inside the warp's area) of lane `lane4 / 4`'s counter for exponent x
+template <int DT>
+__device__ __forceinline__ uint32_t counter_offset(uint32_t x) {
+    constexpr int Q = HistShape<DT>::kQuads;
+    return ((x & (Q - 1)) << 7) + (x / Q);
+}
+
+template <int DT>
+__device__ __forceinline__ void count_word_pair(uint32_t base, uint32_t w) {
+    // two 16-bit values per 32-bit word
+    constexpr int sh = DT == ENEC_BF16 ? 7 : 10;
+    constexpr uint32_t fm = DT == ENEC_BF16 ? 0xFFu : 0x1Fu;
+    const uint32_t a0 = base + counter_offset<DT>((w >> sh) & fm);
+    sts8(a0, lds8(a0) + 1);
+    const uint32_t a1 = base + counter_offset<DT>((w >> (16 + sh)) & fm);
+    sts8(a1, lds8(a1) + 1);
+}
+
+template <int DT>
+__device__ __forceinline__ void flush_counters(uint32_t warp_base, uint32_t lane, uint32_t* cta_hist) {
+    constexpr int Q = HistShape<DT>::kQuads;
+    __syncwarp();
+    for (uint32_t qd = lane; qd < uint32_t(Q); qd += 32) {
+        uint32_t even = 0, odd = 0;  // 16-bit sums of counter bytes 0|2 and 1|3
+#pragma unroll 8
+        for (uint32_t r = 0; r < 32; ++r) {
+            const uint32_t a = warp_base + qd * 128 + ((r + lane) & 31) * 4;
+            const uint32_t v = lds32(a);
+            even += v & 0x00FF00FFu;
+            odd += (v >> 8) & 0x00FF00FFu;
+            sts32(a, 0);
+        }
+        // counter byte s of quad qd belongs to bin s * Q + qd
+        if (even & 0xFFFFu) atomicAdd(&cta_hist[0 * Q + qd], even & 0xFFFFu);
+        if (odd & 0xFFFFu) atomicAdd(&cta_hist[1 * Q + qd], odd & 0xFFFFu);
+        if (even >> 16) atomicAdd(&cta_hist[2 * Q + qd], even >> 16);
+        if (odd >> 16) atomicAdd(&cta_hist[3 * Q + qd], odd >> 16);
+    }
+    __syncwarp();
+}
+
+__host__ __device__ inline int bit_width_u32(uint32_t v) {
+    int w = 0;
+    while (v) { ++w; v >>= 1; }
+    return w;
+}
+
+// Eq. 1 with the logarithms of 0 and 1 read as 0 and the result kept inside 1..E.
+__host__ __device__ inline int width_eq1(int b, int l, int h, int E) {
+    const int pos = bit_width_u32(uint32_t(b - l));
+    const int d = h - b;
+    const int neg = d <= 1 ? 0 : bit_width_u32(uint32_t(d - 1));
+    int n = (pos > neg ? pos : neg) + 1;
+    if (n > E) n = E;
+    return n;
+}
+
+// Sec. 5.5 phases 2 and 3 on the finished histogram; all kHistThreads threads of one CTA.
+template <int DT>
+__device__ void parameter_search(EncodeControl* ctl) {
+    constexpr int E = HistShape<DT>::E;
+    constexpr int kBins = 1 << E;
+    __shared__ unsigned long long s_hist[256];
+    __shared__ unsigned long long s_key[kHistThreads / 32];
+    __shared__ unsigned long long s_width_count[9];
+    __shared__ int s_lo, s_hi, s_b, s_n;
+    const uint32_t tid = threadIdx.x;
+    s_hist[tid] = tid < uint32_t(kBins) ? ld_relaxed_u64(&ctl->hist[tid]) : 0ull;
+    if (tid < 9) s_width_count[tid] = 0;
+    if (tid == 0) { s_lo = kBins; s_hi = -1; }
+    __syncthreads();
+    if (s_hist[tid]) { atomicMin(&s_lo, int(tid)); atomicMax(&s_hi, int(tid)); }
+    __syncthreads();
+    const int l = s_lo, h = s_hi;
+    // phase 2: every candidate b in [l, h]; cost = sum c[x] * y (Eq. 3 times N); smallest (cost, n, b)
+    unsigned long long key = ~0ull;
+    if (int(tid) >= l && int(tid) <= h) {
+        const int b = int(tid);
+        const int n = width_eq1(b, l, h, E);
+        const uint32_t nmask = (1u << n) - 1;
+        unsigned long long cost = 0;
+        for (int x = l; x <= h; ++x) cost += s_hist[x] * (unsigned long long)(uint32_t(b - x) & nmask);
+        key = (cost << 12) | (unsigned long long)(n << 8) | (unsigned long long)b;  // cost < 2^44
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, key, d);
+        key = o < key ? o : key;
+    }
+    if ((tid & 31) == 0) s_key[tid >> 5] = key;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long best = s_key[0];
+        for (int i = 1; i < kHistThreads / 32; ++i) best = s_key[i] < best ? s_key[i] : best;
+        s_b = int(best & 0xFF);
+        s_n = int((best >> 8) & 0xF);
+    }
+    __syncthreads();
+    const int b = s_b, n = s_n;
+    // phase 3: elements per bit width of y, then Eq. 4 at L = 16 for every m
+    if (int(tid) >= l && int(tid) <= h && s_hist[tid]) {
+        const uint32_t y = uint32_t(b - int(tid)) & ((1u << n) - 1);
+        atomicAdd(&s_width_count[bit_width_u32(y)], s_hist[tid]);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long total = 0;
+        for (int w = 0; w <= 8; ++w) total += s_width_count[w];
+        unsigned long long cnt = s_width_count[0];
+        int best_m = 1;
+        double best_bits = 0.0;
+        for (int m = 1; m <= n; ++m) {
+            cnt += s_width_count[m];
+            // plain IEEE double, one rounding per operation, no fused multiply-add
+            const double p = __ddiv_rn(__ull2double_rn(cnt), __ull2double_rn(total));
+            const double p2 = __dmul_rn(p, p);
+            const double p4 = __dmul_rn(p2, p2);
+            const double p8 = __dmul_rn(p4, p4);
+            const double p16 = __dmul_rn(p8, p8);
+            const double saving = __dmul_rn(double(m - n), p16);
+            const double bits = __dadd_rn(__dadd_rn(double(n), 0.0625), saving);  // 1/L + n + (m - n) p^L
+            if (m == 1 || bits < best_bits) { best_m = m; best_bits = bits; }
+        }
+        ctl->b = b;
+        ctl->n = n;
+        ctl->m = best_m;
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kHistThreads, 3)
+enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeControl* ctl) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ uint32_t cta_hist[256];
+    __shared__ int s_last;
+    constexpr int kWarpBytes = HistShape<DT>::kWarpBytes;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t warp_base = smem_u32(smem) + warp * kWarpBytes;
+    const uint32_t base = warp_base + lane * 4;
+    for (uint32_t i = tid; i < uint32_t(kWarpBytes / 4) * (kHistThreads / 32); i += kHistThreads)
+        reinterpret_cast<uint32_t*>(smem)[i] = 0;
+    cta_hist[tid] = 0;
+    __syncthreads();
+
+    const uint64_t nchunks = count >> 3;  // 16-byte loads of eight values
+    const uint4* in4 = reinterpret_cast<const uint4*>(in);
+    const uint64_t stride = uint64_t(gridDim.x) * kHistThreads;
+    uint32_t since_flush = 0;
+    for (uint64_t first = uint64_t(blockIdx.x) * kHistThreads + (tid & ~31u); first < nchunks; first += stride) {
+        const uint64_t i = first + lane;
+        if (i < nchunks) {
+            const uint4 v = in4[i];  // default caching: the encode pass reads the tensor again
+            count_word_pair<DT>(base, v.x);
+            count_word_pair<DT>(base, v.y);
+            count_word_pair<DT>(base, v.z);
+            count_word_pair<DT>(base, v.w);
+        }
+        if (++since_flush == 31) {
+            flush_counters<DT>(warp_base, lane, cta_hist);
+            since_flush = 0;
+        }
+    }
+    flush_counters<DT>(warp_base, lane, cta_hist);
+    if (blockIdx.x == 0 && tid == 0) {  // the last count mod 8 values
+        constexpr int sh = DT == ENEC_BF16 ? 7 : 10;
+        for (uint64_t e = nchunks << 3; e < count; ++e)
+            atomicAdd(&cta_hist[(in[e] >> sh) & (HistShape<DT>::kBins - 1)], 1u);
+    }
+    __syncthreads();
+    if (cta_hist[tid]) atomicAdd(&ctl->hist[tid], (unsigned long long)cta_hist[tid]);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&ctl->hist_done, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    parameter_search<DT>(ctl);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Algorithm 2 on packed bytes (forward). A thread that owns the eight lanes j..j+7 of the deepest level
+// owns, at every level, whole runs of eight consecutive lanes: the 64 elements {j + c N/8 + i : c, i < 8}.
+// Their fields are merged into 16-bit lanes kept as a low and a high byte plane; the low bytes are the
+// level's normalised bytes, the high bytes its residue, packed again by the next level.
+// ---------------------------------------------------------------------------------------------------
+// ORs the w-bit fields v (one per byte, no other bits set) into the 16-bit lanes (lo | hi << 8) at bit s.
+__device__ __forceinline__ void insert_bits(uint32_t& lo, uint32_t& hi, uint32_t v, int s, int w) {
+    if (s + w <= 8) {
+        lo |= v << s;
+    } else if (s >= 8) {
+        hi |= v << (s - 8);
+    } else {
+        const uint32_t keep = 0xFFu >> s;  // bits of a field that stay in the low byte
+        lo |= (v & rep4(keep)) << s;
+        hi |= (v >> (8 - s)) & rep4(((1u << w) - 1) >> (8 - s));
+    }
+}
+
+// in[e] (e < 2^LOG_UNITS) = W_IN-bit fields of the eight elements j + e * n8 + (0..7) of this level.
+// Normalised bytes are written in their order before the final fold: byte i of the plane at S + i.
+template <int W_IN, int LOG_UNITS>
+__device__ __forceinline__ void pack_plane_level(uint32_t S, uint32_t nb_off, uint32_t j, uint32_t n8,
+                                                 const uint2 (&in)[1 << LOG_UNITS]) {
+    constexpr int F = folds_for(W_IN);
+    static_assert(F <= LOG_UNITS, "lane runs must stay whole");
+    constexpr int W = W_IN << F;
+    constexpr int LOG_LANES = LOG_UNITS - F;
+    constexpr int NL = 1 << LOG_LANES;
+    constexpr int RES = W - 8;
+    uint2 R[NL];
+#pragma unroll
+    for (int c = 0; c < NL; ++c) {
+        uint2 V = make_uint2(0, 0);
+        R[c] = make_uint2(0, 0);
+#pragma unroll
+        for (int q = 0; q < (1 << F); ++q) {
+            const int e = c + q * NL;
+            const int s = W_IN * bitrev(q, F);
+            insert_bits(V.x, R[c].x, in[e].x, s, W_IN);
+            insert_bits(V.y, R[c].y, in[e].y, s, W_IN);
+        }
+        sts64(S + nb_off + j + c * n8, V);
+    }
+    if constexpr (RES > 0) pack_plane_level<RES, LOG_LANES>(S, nb_off + NL * n8, j, n8, R);
+}
+
+template <int A>
+__device__ __forceinline__ void pack_plane(uint32_t S, uint32_t j, uint32_t N, const uint2 (&v)[8]) {
+    pack_plane_level<A, 3>(S, 0, j, N >> 3, v);
+}
+
+__device__ __forceinline__ void pack_plane_any(int a, uint32_t S, uint32_t j, uint32_t N, const uint2 (&v)[8]) {
+    switch (a) {
+        case 1: pack_plane<1>(S, j, N, v); break;
+        case 2: pack_plane<2>(S, j, N, v); break;
+        case 3: pack_plane<3>(S, j, N, v); break;
+        case 4: pack_plane<4>(S, j, N, v); break;
+        case 5: pack_plane<5>(S, j, N, v); break;
+        case 6: pack_plane<6>(S, j, N, v); break;
+        case 7: pack_plane<7>(S, j, N, v); break;
+        default: pack_plane<8>(S, j, N, v); break;
+    }
+}
+
+// Final fold of Algorithm 2: output byte 2i = normalised byte i, 2i + 1 = normalised byte i + T/2.
+// Reads the plane (T bytes at shared address S) and writes it folded to `dst`, 16 bytes per step.
+__device__ __forceinline__ void fold_plane_out(uint32_t S, uint32_t T, uint8_t* dst, uint32_t tid) {
+    const uint32_t thalf = T >> 1;
+    for (uint32_t u = tid; u < (thalf >> 3); u += kEncodeThreads) {
+        const uint2 lo = lds64(S + 8 * u);
+        const uint2 hi = lds64(S + thalf + 8 * u);
+        uint4 w;
+        w.x = prmt(lo.x, hi.x, 0x5140u);
+        w.y = prmt(lo.x, hi.x, 0x7362u);
+        w.z = prmt(lo.y, hi.y, 0x5140u);
+        w.w = prmt(lo.y, hi.y, 0x7362u);
+        *reinterpret_cast<uint4*>(dst + 16 * u) = w;
+    }
+}
+
+// ---- wide-group records: Algorithm 2 with N = 16 and H bits per value -> H 16-bit words ---------------
+// Same scheme with runs of two lanes. in[e] = fields of elements 2e, 2e + 1 in bytes 0 and 1.
+template <int H, int W_IN, int LOG_UNITS, int NB_OFF>
+__device__ __forceinline__ void pack_record_level(uint32_t (&q)[H], const uint32_t (&in)[1 << LOG_UNITS]) {
+    constexpr int F = folds_for(W_IN);
+    static_assert(F <= LOG_UNITS, "lane runs must stay whole");
+    constexpr int W = W_IN << F;
+    constexpr int LOG_LANES = LOG_UNITS - F;
+    constexpr int NL = 1 << LOG_LANES;
+    constexpr int RES = W - 8;
+    uint32_t R[NL];
+#pragma unroll
+    for (int c = 0; c < NL; ++c) {
+        uint32_t V = 0;
+        R[c] = 0;
+#pragma unroll
+        for (int k = 0; k < (1 << F); ++k) {
+            const int e = c + k * NL;
+            insert_bits(V, R[c], in[e], W_IN * bitrev(k, F), W_IN);
+        }
+        // normalised bytes i0, i0 + 1 of the record; byte i sits at 2i (i < H) or 2(i - H) + 1
+        const int i0 = NB_OFF + 2 * c;
+        const int pa = i0 < H ? 2 * i0 : 2 * (i0 - H) + 1;
+        const int pb = (i0 + 1) < H ? 2 * (i0 + 1) : 2 * (i0 + 1 - H) + 1;
+        q[pa >> 1] |= (V & 0xFFu) << (8 * (pa & 1));
+        q[pb >> 1] |= ((V >> 8) & 0xFFu) << (8 * (pb & 1));
+    }
+    if constexpr (RES > 0) pack_record_level<H, RES, LOG_LANES, NB_OFF + 2 * NL>(q, R);
+}
+
+// v = the sixteen H-bit values of a group, one per byte, element order; the record goes to shared
+// address `dst` (2-byte aligned) as H 16-bit words.
+template <int H>
+__device__ __forceinline__ void pack_record(uint4 v, uint32_t dst) {
+    uint32_t in[8] = {v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16,
+                      v.z & 0xFFFFu, v.z >> 16, v.w & 0xFFFFu, v.w >> 16};
+    uint32_t q[H];
+#pragma unroll
+    for (int i = 0; i < H; ++i) q[i] = 0;
+    pack_record_level<H, H, 3, 0>(q, in);
+#pragma unroll
+    for (int i = 0; i < H; ++i) sts16(dst + 2 * i, q[i]);
+}
+
+__device__ __forceinline__ void pack_record_any(int hbits, uint4 v, uint32_t dst) {
+    switch (hbits) {
+        case 1: pack_record<1>(v, dst); break;
+        case 2: pack_record<2>(v, dst); break;
+        case 3: pack_record<3>(v, dst); break;
+        case 4: pack_record<4>(v, dst); break;
+        case 5: pack_record<5>(v, dst); break;
+        case 6: pack_record<6>(v, dst); break;
+        default: pack_record<7>(v, dst); break;
+    }
+}
+
+// Where bit q of element e of a plane of N elements of `a` bits ends up: byte `pos` of the packed plane,
+// bit `bit` (Algorithm 2 followed for one bit; used for blocks shorter than 128 elements).
+__device__ inline void alg2_locate(uint32_t N, int a, uint32_t e, int q, uint32_t& pos, int& bit) {
+    const uint32_t thalf = (N * uint32_t(a)) >> 4;
+    int width = a, p = q;
+    uint32_t length = N, idx = e, off = 0;
+    while (true) {
+        while (length > 1 && width < 8) {
+            length >>= 1;
+            if (idx >= length) { idx -= length; p += width; }
+            width <<= 1;
+        }
+        if (p < 8) break;
+        p -= 8;
+        width -= 8;
+        off += length;
+    }
+    const uint32_t i = off + idx;
+    pos = i < thalf ? 2 * i : 2 * (i - thalf) + 1;
+    bit = p;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Split and transform on packed bytes.
+// ---------------------------------------------------------------------------------------------------
+struct Split4 {
+    uint32_t x;   // exponent fields of four values, one per byte
+    uint32_t sm;  // bf16: sign << 7 | mantissa ; fp16: mantissa bits 7..0
+    uint32_t hs;  // fp16: sign << 2 | mantissa bits 9..8
+};
+
+template <int DT>
+__device__ __forceinline__ Split4 split4(uint32_t w0, uint32_t w1) {
+    const uint32_t lo = prmt(w0, w1, 0x6420u);  // low bytes of the four 16-bit words
+    const uint32_t hi = prmt(w0, w1, 0x7531u);  // high bytes
+    Split4 s;
+    if (DT == ENEC_BF16) {
+        s.x = ((hi << 1) & 0xFEFEFEFEu) | ((lo >> 7) & 0x01010101u);
+        s.sm = (hi & 0x80808080u) | (lo & 0x7F7F7F7Fu);
+        s.hs = 0;
+    } else {
+        s.x = (hi >> 2) & 0x1F1F1F1Fu;
+        s.sm = lo;
+        s.hs = ((hi >> 5) & 0x04040404u) | (hi & 0x03030303u);
+    }
+    return s;
+}
+
+struct TransformCtx {
+    uint32_t b4_or_h;   // rep4(b) | 0x80808080
+    uint32_t b4;        // rep4(b)
+    uint32_t nmask4;    // rep4(2^n - 1)
+    uint32_t s4;        // rep4(2^(n-1))
+    uint32_t emask4;    // rep4(2^E - 1)
+    int n, E;
+};
+
+// b - x modulo 256 in every byte
+__device__ __forceinline__ uint32_t bytewise_b_minus(const TransformCtx& t, uint32_t x) {
+    return (t.b4_or_h - (x & 0x7F7F7F7Fu)) ^ ((t.b4 ^ ~x) & 0x80808080u);
+}
+
+// Bytes whose exponent is not reproduced by (b, n): x != (b - sext_n(y)) mod 2^E. Non-zero = some byte fails.
+__device__ __forceinline__ uint32_t lossy_bytes(const TransformCtx& t, uint32_t d, uint32_t y) {
+    if (t.n == t.E) return 0;
+    // sext_n(y) = (y ^ s) - s per byte; (y ^ s) < 128 because n < 8
+    const uint32_t sext = (((y ^ t.s4) | 0x80808080u) - t.s4) ^ 0x80808080u;
+    return (sext ^ d) & t.emask4;
+}
+
+// ---------------------------------------------------------------------------------------------------
+struct EncodeShared {
+    uint32_t mask[32];     // the block's group mask, bit g = group g is wide
+    uint32_t prefix[32];   // wide groups before each mask word
+    uint32_t group_or[8];  // short blocks: OR of y per group
+    uint32_t block;        // ticket
+    uint32_t wide;         // A_k
+    uint32_t before;       // P_k
+    uint32_t poisoned;
+};
+
+// Blocks shorter than 128 elements (16, 32 or 64): one element per thread, bits placed one by one.
+template <int DT>
+__device__ __noinline__ int encode_short_block(const uint16_t* in, uint32_t N, uint32_t real, const TransformCtx& tc,
+                                               int b, int n, int m, int check, uint8_t* out_sm, uint8_t* out_low,
+                                               uint8_t* out_smhi, uint8_t* out_mask, EncodeShared* sh,
+                                               uint32_t* s_low, uint32_t* s_hi3, uint32_t* s_rec) {
+    const uint32_t tid = threadIdx.x;
+    const int hbits = n - m;
+    if (tid < 32) sh->mask[tid] = 0;
+    if (tid < 8) sh->group_or[tid] = 0;
+    if (tid < 16) { s_low[tid] = 0; s_rec[tid] = 0; }
+    if (tid < 8) s_hi3[tid] = 0;
+    __syncthreads();
+    int bad = 0;
+    uint32_t y = 0;
+    if (tid < N) {
+        const uint32_t w = tid < real ? in[tid] : 0;
+        uint32_t x, sm, hs = 0;
+        if (DT == ENEC_BF16) { x = (w >> 7) & 0xFF; sm = ((w >> 8) & 0x80) | (w & 0x7F); }
+        else { x = (w >> 10) & 0x1F; sm = w & 0xFF; hs = ((w >> 13) & 4) | ((w >> 8) & 3); }
+        if (tid < real) {
+            y = uint32_t(b - int(x)) & ((1u << n) - 1);
+            if (check && n < tc.E) {
+                const int v = (y >> (n - 1)) ? int(y) - (1 << n) : int(y);
+                bad = (uint32_t(b - v) & ((1u << tc.E) - 1)) != x;
+            }
+            out_sm[tid] = uint8_t(sm);
+        } else if (tid < uint32_t(align16(real))) {
+            out_sm[tid] = 0;
+        }
+        atomicOr(&sh->group_or[tid >> 4], y);
+        for (int q = 0; q < m; ++q)
+            if ((y >> q) & 1) {
+                uint32_t pos; int bit;
+                alg2_locate(N, m, tid, q, pos, bit);
+                atomicOr(&s_low[pos >> 2], 1u << (8 * (pos & 3) + bit));
+            }
+        if (DT == ENEC_FP16)
+            for (int q = 0; q < 3; ++q)
+                if ((hs >> q) & 1) {
+                    uint32_t pos; int bit;
+                    alg2_locate(N, 3, tid, q, pos, bit);
+                    atomicOr(&s_hi3[pos >> 2], 1u << (8 * (pos & 3) + bit));
+                }
+    }
+    __syncthreads();
+    const bool wide = tid < N && (sh->group_or[tid >> 4] >> m) != 0;
+    if (wide && (tid & 15) == 0) atomicOr(&sh->mask[0], 1u << (tid >> 4));
+    __syncthreads();
+    if (wide && hbits > 0) {
+        const uint32_t rank = __popc(sh->mask[0] & ((1u << (tid >> 4)) - 1));
+        const uint32_t hv = y >> m;
+        for (int q = 0; q < hbits; ++q)
+            if ((hv >> q) & 1) {
+                uint32_t pos; int bit;
+                alg2_locate(16, hbits, tid & 15, q, pos, bit);
+                pos += rank * 2 * hbits;
+                atomicOr(&s_rec[pos >> 2], 1u << (8 * (pos & 3) + bit));
+            }
+    }
+    // planes out, padded to 16 bytes with zeros
+    const uint32_t low_words = uint32_t(align16(N * uint32_t(m) / 8)) / 4;
+    if (tid < low_words) reinterpret_cast<uint32_t*>(out_low)[tid] = s_low[tid];
+    if (tid < 4) reinterpret_cast<uint32_t*>(out_mask)[tid] = tid == 0 ? sh->mask[0] : 0;
+    if (DT == ENEC_FP16) {
+        const uint32_t hi_words = uint32_t(align16(N * 3 / 8)) / 4;
+        if (tid < hi_words) reinterpret_cast<uint32_t*>(out_smhi)[tid] = s_hi3[tid];
+    }
+    return bad;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kEncodeThreads, 4)
+enec_encode_kernel(EncodeJob job, int* status) {
+    constexpr int E = DT == ENEC_BF16 ? 8 : 5;
+    __shared__ __align__(16) uint8_t s_low[kBlockElems];                              // normalised bytes, low plane
+    __shared__ __align__(16) uint8_t s_hi3[DT == ENEC_FP16 ? kBlockElems * 3 / 8 : 32];  // fp16 sign/mantissa-high plane
+    __shared__ __align__(16) uint8_t s_rec[kGroupsPerBlock * 14];                     // records of the block, rank order
+    __shared__ EncodeShared sh;
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        sh.block = atomicAdd(&job.ctl->ticket, 1u);
+        sh.poisoned = 0;
+    }
+    __syncthreads();
+    const uint32_t k = sh.block;
+
+    int b = job.b, n = job.n, m = job.m;
+    if (job.from_search) { b = job.ctl->b; n = job.ctl->n; m = job.ctl->m; }
+    const int hbits = n - m;
+    const Geometry g = make_geometry(job.count);
+    const Sections sec = make_sections(DT, job.count, g, n, m, 0);
+    if (k >= g.nblocks) return;
+    const bool last = k + 1 == g.nblocks;
+    const uint32_t N = last ? g.tail_padded : kBlockElems;
+    const uint32_t real = last ? g.tail_real : kBlockElems;
+    const uint16_t* in = job.in + uint64_t(k) * kBlockElems;
+    uint8_t* out_sm = job.out + sec.sm + uint64_t(k) * kBlockElems;
+    uint8_t* out_low = job.out + sec.low + uint64_t(k) * (kBlockElems / 8) * uint32_t(m);
+    uint8_t* out_smhi = job.out + sec.smhi + uint64_t(k) * (kBlockElems / 8) * 3;
+    uint8_t* out_mask = job.out + sec.mask + uint64_t(k) * (kGroupsPerBlock / 8);
+
+    TransformCtx tc;
+    tc.b4 = rep4(uint32_t(b));
+    tc.b4_or_h = tc.b4 | 0x80808080u;
+    tc.nmask4 = rep4((1u << n) - 1);
+    tc.s4 = rep4(1u << (n - 1));
+    tc.emask4 = rep4((1u << E) - 1);
+    tc.n = n;
+    tc.E = E;
+
+    int bad = 0;
+    uint2 y[8];
+    uint32_t wide_bits = 0;  // bit c: the group of run c is wide
+    const bool fast = N == kBlockElems;
+    // fast path: lanes l and l + 16 share a group, so a ballot's low half is the mask of sixteen groups
+    const uint32_t perm = fast ? (warp * 32 + 2 * (lane & 15) + (lane >> 4)) : tid;
+    const uint32_t pair_delta = fast ? 16 : 1;
+    const bool first_of_pair = fast ? lane < 16 : (lane & 1) == 0;
+    const uint32_t n8 = N >> 3;
+    const uint32_t j = 8 * perm;
+    const bool active = N >= 128 && perm < (N >> 6);
+
+    if (N >= 128) {
+        if (!fast) {
+            if (tid < 32) sh.mask[tid] = 0;
+            __syncthreads();
+        }
+        uint4 raw[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint32_t e0 = c * n8 + j;
+            raw[c] = make_uint4(0, 0, 0, 0);
+            if (active) {
+                if (e0 + 8 <= real) {
+                    raw[c] = __ldcs(reinterpret_cast<const uint4*>(in + e0));
+                } else if (e0 < real) {
+                    uint32_t v[4] = {0, 0, 0, 0};
+                    for (uint32_t i = 0; e0 + i < real; ++i) v[i >> 1] |= uint32_t(in[e0 + i]) << (16 * (i & 1));
+                    raw[c] = make_uint4(v[0], v[1], v[2], v[3]);
+                }
+            }
+        }
+        uint2 hs[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint32_t e0 = c * n8 + j;
+            const Split4 s0 = split4<DT>(raw[c].x, raw[c].y);
+            const Split4 s1 = split4<DT>(raw[c].z, raw[c].w);
+            const uint32_t d0 = bytewise_b_minus(tc, s0.x), d1 = bytewise_b_minus(tc, s1.x);
+            y[c] = make_uint2(d0 & tc.nmask4, d1 & tc.nmask4);
+            hs[c] = make_uint2(s0.hs, s1.hs);
+            if (active && e0 + 8 > real) {  // padding elements carry y = 0
+                const uint32_t valid = e0 < real ? real - e0 : 0;
+                const uint32_t k0 = valid >= 4 ? 0xFFFFFFFFu : (1u << (8 * valid)) - 1;
+                const uint32_t k1 = valid >= 8 ? 0xFFFFFFFFu : valid > 4 ? (1u << (8 * (valid - 4))) - 1 : 0;
+                y[c].x &= k0;
+                y[c].y &= k1;
+            }
+            if (!active) y[c] = make_uint2(0, 0);
+            if (job.check && active && e0 + 8 <= real)
+                bad |= (lossy_bytes(tc, d0, y[c].x) | lossy_bytes(tc, d1, y[c].y)) != 0;
+            else if (job.check && active && e0 < real) {
+                const uint32_t valid = real - e0;
+                const uint32_t k0 = valid >= 4 ? 0xFFFFFFFFu : (1u << (8 * valid)) - 1;
+                const uint32_t k1 = valid > 4 ? (1u << (8 * (valid - 4))) - 1 : 0;
+                bad |= ((lossy_bytes(tc, d0, y[c].x) & k0) | (lossy_bytes(tc, d1, y[c].y) & k1)) != 0;
+            }
+            if (active && e0 < uint32_t(align16(real)))
+                __stcs(reinterpret_cast<uint2*>(out_sm + e0), make_uint2(s0.sm, s1.sm));
+            uint32_t o = y[c].x | y[c].y;
+            o |= o >> 16;
+            o |= o >> 8;
+            o |= __shfl_xor_sync(0xFFFFFFFFu, o, pair_delta);
+            const bool wide = ((o & 0xFFu) >> m) != 0;
+            wide_bits |= uint32_t(wide) << c;
+            if (fast) {
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, wide);
+                if (lane == 0) reinterpret_cast<uint16_t*>(sh.mask)[c * 8 + warp] = uint16_t(bal);
+            } else if (wide && first_of_pair && active) {
+                const uint32_t grp = e0 >> 4;
+                atomicOr(&sh.mask[grp >> 5], 1u << (grp & 31));
+            }
+        }
+        if (active) {
+            uint2 ylow[8];
+            const uint32_t lowmask4 = rep4((1u << m) - 1);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) ylow[c] = make_uint2(y[c].x & lowmask4, y[c].y & lowmask4);
+            pack_plane_any(m, smem_u32(s_low), j, N, ylow);
+            if (DT == ENEC_FP16) pack_plane<3>(smem_u32(s_hi3), j, N, hs);
+        }
+    } else {
+        bad = encode_short_block<DT>(in, N, real, tc, b, n, m, job.check, out_sm, out_low, out_smhi, out_mask, &sh,
+                                     reinterpret_cast<uint32_t*>(s_low), reinterpret_cast<uint32_t*>(s_hi3),
+                                     reinterpret_cast<uint32_t*>(s_rec));
+    }
+    const int any_bad = __syncthreads_or(bad);
+
+    // wide groups before each mask word, and in the block
+    if (warp == 0) {
+        const uint32_t mw = sh.mask[lane];
+        uint32_t incl = __popc(mw);
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= uint32_t(d)) incl += t;
+        }
+        sh.prefix[lane] = incl - __popc(mw);
+        if (lane == 31) {
+            sh.wide = incl;
+            if (any_bad) {
+                report(status, ENEC_ERR_PARAMS_NOT_LOSSLESS);
+                atomicOr(&job.ctl->error, 1u);
+            }
+            __threadfence();
+            // publish this block's count at once; block 0 knows its prefix already
+            st_relaxed_u64(&job.state[k], (k == 0 ? kStatePrefix : kStateAggregate) | incl);
+        }
+    }
+    __syncthreads();
+    const uint32_t wide_count = sh.wide;
+
+    if (N >= 128) {
+        fold_plane_out(smem_u32(s_low), N * uint32_t(m) / 8, out_low, tid);
+        if (DT == ENEC_FP16) fold_plane_out(smem_u32(s_hi3), N * 3 / 8, out_smhi, tid);
+        const uint32_t mask_vecs = uint32_t(align16(((N >> 4) + 7) / 8)) / 16;
+        if (tid < mask_vecs)
+            reinterpret_cast<uint4*>(out_mask)[tid] = reinterpret_cast<const uint4*>(sh.mask)[tid];
+        // records of wide groups into shared memory, rank order
+        if (hbits > 0) {
+            const uint32_t hmask4 = rep4(0xFFu >> m);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t h0 = (y[c].x >> m) & hmask4, h1 = (y[c].y >> m) & hmask4;
+                const uint32_t p0 = __shfl_down_sync(0xFFFFFFFFu, h0, pair_delta);
+                const uint32_t p1 = __shfl_down_sync(0xFFFFFFFFu, h1, pair_delta);
+                if (((wide_bits >> c) & 1) && first_of_pair && active) {
+                    const uint32_t grp = (c * n8 + j) >> 4;
+                    const uint32_t rank = sh.prefix[grp >> 5] + __popc(sh.mask[grp >> 5] & ((1u << (grp & 31)) - 1));
+                    pack_record_any(hbits, make_uint4(h0, h1, p0, p1), smem_u32(s_rec) + rank * 2 * hbits);
+                }
+            }
+        }
+    }
+
+    // block-offset prefix sum: look back over the predecessors' state words (warp 0)
+    if (warp == 0 && k > 0) {
+        uint32_t before = 0;
+        int64_t pos = int64_t(k) - 1;
+        int outcome = 0;  // 1 = done, 2 = poisoned, 3 = gave up
+        uint32_t polls = 0;
+        while (outcome == 0) {
+            const int64_t idx = pos - lane;
+            unsigned long long st = idx >= 0 ? ld_relaxed_u64(&job.state[idx]) : kStatePrefix;
+            const uint32_t kind = uint32_t(st >> 62);
+            const uint32_t prefix_lanes = __ballot_sync(0xFFFFFFFFu, kind == 2);
+            const uint32_t empty_lanes = __ballot_sync(0xFFFFFFFFu, kind == 0);
+            const uint32_t poison_lanes = __ballot_sync(0xFFFFFFFFu, kind == 3);
+            const uint32_t first = prefix_lanes ? uint32_t(__ffs(prefix_lanes)) - 1 : 32;
+            const uint32_t needed = first == 32 ? 0xFFFFFFFFu : (2u << first) - 1;  // lanes 0..first
+            if (poison_lanes & needed) { outcome = 2; break; }
+            if (empty_lanes & needed) {
+                if (++polls > (1u << 20)) { outcome = 3; break; }
+                if (polls > 8) __nanosleep(200);
+                continue;
+            }
+            uint32_t v = (needed >> lane) & 1 ? uint32_t(st) : 0;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+            before += v;
+            if (first < 32) outcome = 1;
+            else pos -= 32;
+        }
+        if (lane == 0) {
+            if (outcome == 1) {
+                sh.before = before;
+                __threadfence();
+                st_relaxed_u64(&job.state[k], kStatePrefix | (unsigned long long)(before + wide_count));
+            } else {
+                if (outcome == 3) report(status, ENEC_ERR_TIMEOUT);
+                atomicOr(&job.ctl->error, 1u);
+                __threadfence();
+                st_relaxed_u64(&job.state[k], kStatePoison);
+                sh.poisoned = 1;
+                sh.before = 0;
+            }
+        }
+    } else if (tid == 0 && k == 0) {
+        sh.before = 0;
+    }
+    __syncthreads();
+    const uint32_t before = sh.before;
+    const bool poisoned = sh.poisoned != 0;
+
+    uint32_t* table = reinterpret_cast<uint32_t*>(job.out + sec.table);
+    if (!poisoned) {
+        // records to their place in the stream: record r of the tensor at r * 2 * hbits
+        uint16_t* dst = reinterpret_cast<uint16_t*>(job.out + sec.high + uint64_t(before) * 2 * uint32_t(hbits));
+        const uint16_t* src = reinterpret_cast<const uint16_t*>(s_rec);
+        for (uint32_t i = tid; i < wide_count * uint32_t(hbits); i += kEncodeThreads) dst[i] = src[i];
+        if (tid == 0) table[k] = before;
+    }
+    if (last && tid == 0) {
+        const uint32_t a_total = before + wide_count;
+        const uint64_t high_bytes = uint64_t(a_total) * 2 * uint32_t(hbits);
+        const uint64_t total = sec.high + align16(high_bytes);
+        __threadfence();
+        const bool failed = poisoned || ld_relaxed_u32(&job.ctl->error) != 0;
+        Header hd;
+        hd.magic = failed ? 0 : kMagic;
+        hd.version = kVersion;
+        hd.dtype = DT;
+        hd.pad0 = 0;
+        hd.count = job.count;
+        hd.block = kBlockElems;
+        hd.b = uint8_t(b); hd.n = uint8_t(n); hd.m = uint8_t(m); hd.L = kGroupElems;
+        hd.nblocks = g.nblocks;
+        hd.total_groups = g.total_groups;
+        hd.a_total = a_total;
+        hd.pad1 = 0;
+        hd.total_bytes = total;
+        hd.pad2[0] = hd.pad2[1] = 0;
+        *reinterpret_cast<Header*>(job.out) = hd;
+        if (!poisoned) {
+            table[g.nblocks] = a_total;
+            for (uint64_t i = uint64_t(g.nblocks) + 1; i < align16(4 * (uint64_t(g.nblocks) + 1)) / 4; ++i) table[i] = 0;
+            for (uint64_t p = high_bytes; p < align16(high_bytes); p += 2)
+                *reinterpret_cast<uint16_t*>(job.out + sec.high + p) = 0;
+        }
+        if (job.out_size) *job.out_size = failed ? 0ull : total;
+    }
+}
+
+// Stream of an empty tensor: header and a one-entry table.
+__global__ void enec_encode_empty_kernel(uint8_t* out, int dt, int b, int n, int m, unsigned long long* out_size) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    Header hd;
+    hd.magic = kMagic;
+    hd.version = kVersion;
+    hd.dtype = uint8_t(dt);
+    hd.pad0 = 0;
+    hd.count = 0;
+    hd.block = kBlockElems;
+    hd.b = uint8_t(b); hd.n = uint8_t(n); hd.m = uint8_t(m); hd.L = kGroupElems;
+    hd.nblocks = 0;
+    hd.total_groups = 0;
+    hd.a_total = 0;
+    hd.pad1 = 0;
+    hd.total_bytes = kHeaderBytes + 16;
+    hd.pad2[0] = hd.pad2[1] = 0;
+    *reinterpret_cast<Header*>(out) = hd;
+    *reinterpret_cast<uint4*>(out + kHeaderBytes) = make_uint4(0, 0, 0, 0);
+    if (out_size) *out_size = kHeaderBytes + 16;
+}
+
+}  // namespace enec
