@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the ENEC codec on B200: decompress / compress GB/s (uncompressed bytes) and compression ratio on
+a seeded synthetic Llama-3-8B-shaped bf16 weight set.
+
+One step = one pass of the whole hot path over the set: enec_compress (histogram, parameter search, split,
+transform, group widths, Algorithm 2 packing, block-offset prefix sum) of every tensor, then enec_decompress
+(unpack, reconstruct) of every tensor, tensor by tensor on one stream.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama8b|layer|tensor] [--impl reference]
+
+Prints one JSON line (rank 0). `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "bf16 weight decompress GB/s (uncompressed bytes); compress GB/s and compression ratio alongside"
+WORKLOADS = {
+    "llama8b": (3, "full 32-layer Llama-3-8B-shaped bf16 weight set, 291 tensors, 16.06 GB"),
+    "layer": (2, "one Llama-3-8B-shaped decoder layer in bf16, 9 tensors, 436 MB"),
+    "tensor": (1, "one bf16 tensor 1024x4096, 8 MB"),
+}
+SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+
+def measured_peak_gbs():
+    """HBM copy bandwidth measured on this machine (generated file), else the stated fallback."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={SMI_QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if not sm:
+            return None
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_module():
+    sys.path.insert(0, os.path.join(ROOT, "oracle"))
+    import enec_oracle
+    enec_oracle.lib()
+    return enec_oracle
+
+
+def time_oracle(words_list, dt=0):
+    """Single-threaded oracle over a list of numpy uint16 arrays. Returns (compress s, decompress s, raw bytes,
+    stream bytes)."""
+    oracle = oracle_module()
+    tc = td = 0.0
+    raw = comp = 0
+    for w in words_list:
+        t0 = time.perf_counter()
+        s = oracle.compress(w, dt)
+        t1 = time.perf_counter()
+        back = oracle.decompress(s, dt, w.size)
+        t2 = time.perf_counter()
+        assert (back == w).all()
+        tc += t1 - t0
+        td += t2 - t1
+        raw += w.nbytes
+        comp += s.size
+    return tc, td, raw, comp
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores: each step compresses and decompresses a bounded sample of
+    the workload (the four attention projections of one layer, 100 MB of bf16)."""
+    import numpy as np
+    import torch
+    from paper_2604_03298_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, desc = WORKLOADS[args.workload]
+    specs = synth.config_specs(cfg)
+    big = [s for s in specs if s.numel >= 1 << 20]
+    sample = [s for s in big if s.name.split(".")[-1] in ("q", "k", "v", "o")][:4] or big[:1]
+    words = [synth.as_words(synth.make_tensor(s, "cpu")).numpy().view(np.uint16) for s in sample]
+    for _ in range(args.warmup):
+        time_oracle(words[:1])
+    t_comp = t_dec = 0.0
+    t_all0 = time.perf_counter()
+    for _ in range(args.steps):
+        tc, td, raw, comp = time_oracle(words)
+        t_comp += tc
+        t_dec += td
+    t_all = time.perf_counter() - t_all0
+    dec_gbs = raw * args.steps / t_dec / 1e9
+    sample_desc = f"{'+'.join(s.name for s in sample)} of the workload ({raw / 1e6:.0f} MB raw) per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": dec_gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_all / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": desc, "sample": sample_desc},
+        "compress": {"value": raw * args.steps / t_comp / 1e9, "unit": "GB/s"},
+        "compression_ratio": raw / comp,
+        "cpu_baseline": {"value": dec_gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample_desc},
+        "e2e": {"value": dec_gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    import paper_2604_03298_b200 as enec
+    from paper_2604_03298_b200 import runner, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    enec.lib()  # fails loudly if libenec.so is missing
+
+    cfg, desc = WORKLOADS[args.workload]
+    specs = synth.config_specs(cfg)
+    # weak scaling: every rank holds a full copy of the set drawn with its own seeds
+    import dataclasses
+    specs = [dataclasses.replace(s, seed=s.seed + 100003 * rank) for s in specs]
+    raw = [synth.make_tensor(s, "cuda") for s in specs]
+    cs = runner.CodecSet.allocate(raw)
+    raw_bytes = cs.raw_bytes
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # warm-up steps, then one verified round trip (outside the timed region)
+    for _ in range(max(args.warmup, 1)):
+        cs.compress_all()
+        cs.decompress_all()
+    torch.cuda.synchronize()
+    cs.check_status()
+    cs.verify_roundtrip()
+    comp_bytes = cs.compressed_bytes()
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+    launches0 = enec.enec_launch_count()
+    barrier()
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        ev[k][0].record()
+        cs.compress_all()
+        ev[k][1].record()
+        cs.decompress_all()
+        ev[k][2].record()
+    barrier()
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    launches = enec.enec_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    cs.check_status()
+    ms_comp = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    ms_dec = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    ms_step = ev[0][0].elapsed_time(ev[-1][2]) / args.steps
+    ms_comp, ms_dec, ms_step = (runner.max_over_ranks(v) for v in (ms_comp, ms_dec, ms_step))
+    total_raw = runner.sum_over_ranks(raw_bytes)
+    total_comp = runner.sum_over_ranks(comp_bytes)
+    total_launches = int(runner.sum_over_ranks(launches))
+
+    # end to end through host buffers (pinned): host stream -> device -> decompress -> host tensor, and the
+    # compress direction likewise, on one decoder layer of this rank's set
+    layer = [i for i, s in enumerate(specs) if s.name.startswith("l0.") or cfg == 1][:9]
+    h_streams = [torch.empty(int(cs.sizes[i].item()), dtype=torch.uint8).pin_memory() for i in layer]
+    h_raw = [torch.empty(cs.raw[i].numel(), dtype=cs.raw[i].dtype).pin_memory() for i in layer]
+    for h, i in zip(h_streams, layer):
+        h.copy_(cs.streams[i][:h.numel()])
+    for h, i in zip(h_raw, layer):
+        h.copy_(cs.raw[i].reshape(-1))
+    torch.cuda.synchronize()
+    e2e_raw = sum(h.numel() * 2 for h in h_raw)
+    e2e_comp = sum(h.numel() for h in h_streams)
+
+    def e2e_decompress():
+        for h, i in zip(h_streams, layer):
+            cs.streams[i][:h.numel()].copy_(h, non_blocking=True)
+            st = enec.enec_decompress(cs.streams[i], h.numel(), 0 if cs.raw[i].dtype == torch.bfloat16 else 1,
+                                      cs.raw[i].numel(), cs.outs[i], cs.status)
+            assert st == 0
+        for h, i in zip(h_raw, layer):
+            h.copy_(cs.outs[i], non_blocking=True)
+
+    def e2e_compress():
+        for h, i in zip(h_raw, layer):
+            cs.outs[i].copy_(h, non_blocking=True)
+            st = enec.enec_compress(cs.outs[i], 0 if cs.raw[i].dtype == torch.bfloat16 else 1, cs.raw[i].numel(),
+                                    cs.streams[i], cs.streams[i].numel(), cs.sizes[i:i + 1], cs.status)
+            assert st == 0
+        for h, i in zip(h_streams, layer):
+            h.copy_(cs.streams[i][:h.numel()], non_blocking=True)
+
+    def time_e2e(fn):
+        for _ in range(2):
+            fn()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            fn()
+        b.record()
+        barrier()
+        return runner.max_over_ranks(a.elapsed_time(b) / args.steps)
+
+    ms_e2e_dec = time_e2e(e2e_decompress)
+    ms_e2e_comp = time_e2e(e2e_compress)
+    cs.check_status()
+    for h, i in zip(h_raw, layer):  # the host copy of the last decompress must be the tensor
+        assert torch.equal(h.view(torch.int16), cs.raw[i].reshape(-1).view(torch.int16).cpu())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak_gbs()
+    n_dec = len(cs.raw)
+    dec_moved = (raw_bytes + comp_bytes)                       # algorithmic bytes of one decompress pass (this rank)
+    achieved = dec_moved / (ms_dec * 1e-3) / 1e9
+    elems = raw_bytes // 2
+    roofline = {
+        "kernel": "enec_decode_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
+        "algorithmic_bytes_per_launch": dec_moved / n_dec, "launches_per_step": n_dec,
+        "avg_launch_us": ms_dec * 1e3 / n_dec,
+        "traffic": DECODE_DRAM_BYTES_PER_ELEM * elems / n_dec if DECODE_DRAM_BYTES_PER_ELEM else None,
+        "compress": {"achieved": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9,
+                     "frac": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9 / peak,
+                     "note": "algorithmic bytes = read raw once + write stream; the histogram pass reads raw again"},
+    }
+
+    # CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        sample_idx = [i for i, s in enumerate(specs) if s.numel >= 1 << 20][:7]   # one layer's matrices
+        if cfg == 1:
+            sample_idx = [0]
+        words = [cs.raw[i].reshape(-1).view(torch.int16).cpu().numpy().view(np.uint16) for i in sample_idx]
+        tc, td, sraw, scomp = time_oracle(words)
+        gpu_sizes = [int(cs.sizes[i].item()) for i in sample_idx]
+        assert sum(gpu_sizes) == scomp, "GPU and oracle stream sizes differ on the sample"
+        cpu = {"value": sraw / td / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+               "sample": f"{len(sample_idx)} tensors of the workload ({sraw / 1e6:.0f} MB raw), single thread",
+               "compress": {"value": sraw / tc / 1e9, "unit": "GB/s"}, "compression_ratio": sraw / scomp}
+
+    line = {
+        "metric": METRIC, "value": total_raw / (ms_dec * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": desc, "tensors_per_rank": n_dec, "raw_bytes_per_rank": raw_bytes,
+                   "step": "enec_compress of every tensor, then enec_decompress of every tensor, one stream",
+                   "value_is": "uncompressed bytes / time of the step's decompress pass",
+                   "l2": "inputs larger than L2 (each pass streams the whole set)" if raw_bytes > 256e6 else
+                         "set fits in L2: HBM fraction not meaningful",
+                   "sharding": "replica per rank, no collective"},
+        "ms_decompress_per_step": ms_dec, "ms_compress_per_step": ms_comp, "wall_ms_per_step": wall_ms / args.steps,
+        "compress": {"value": total_raw / (ms_comp * 1e-3) / 1e9, "unit": "GB/s"},
+        "roundtrip": {"value": total_raw / (ms_step * 1e-3) / 1e9, "unit": "GB/s"},
+        "compression_ratio": total_raw / total_comp,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_raw * world / (ms_e2e_dec * 1e-3) / 1e9, "unit": "GB/s",
+                "h2d_bytes_per_step": e2e_comp, "d2h_bytes_per_step": e2e_raw,
+                "workload": "one decoder layer of the set: pinned host stream -> device -> enec_decompress -> pinned host",
+                "compress": {"value": e2e_raw * world / (ms_e2e_comp * 1e-3) / 1e9, "unit": "GB/s",
+                             "h2d_bytes_per_step": e2e_raw, "d2h_bytes_per_step": e2e_comp}},
+        "gpu_launches": total_launches,
+        "clocks": clocks,
+        "paper_context": "Ascend 910B2, Llama-3.1-8B bf16: CR 1.36, 376.8 / 219.4 GB/s compress / decompress",
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per element of enec_decode_kernel from the committed ncu capture
+# (profiles/); None until a capture of the current kernel exists.
+DECODE_DRAM_BYTES_PER_ELEM = None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

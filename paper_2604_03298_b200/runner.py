@@ -1,0 +1,109 @@
+"""Host-side driver of the codec over a set of tensors: allocation, one compress pass, one decompress pass,
+sharding of a tensor list over ranks and max-over-ranks timing. Used by the benchmark and the tests.
+
+Every codec step runs in the CUDA library; this module only allocates with torch, marshals through the
+binding and reads status words.
+"""
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import torch
+
+from . import binding as enec
+
+_DT = {torch.bfloat16: enec.BF16, torch.float16: enec.FP16}
+
+
+def shard(items: list, rank: int, world: int) -> list:
+    """Round-robin split of a tensor list over ranks: tensors are independent streams, so a rank needs no
+    data from any other rank (no collective on the data path)."""
+    if not (0 <= rank < world):
+        raise ValueError("rank outside the world")
+    return items[rank::world]
+
+
+def max_over_ranks(value: float, group=None) -> float:
+    """Largest value over all ranks of the process group (the rank's own value without a group)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    dev = "cuda" if dist.get_backend(group) == "nccl" else "cpu"
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, group=None) -> float:
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    dev = "cuda" if dist.get_backend(group) == "nccl" else "cpu"
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+    return float(t.item())
+
+
+@dataclass
+class CodecSet:
+    """Device buffers of a tensor set: raw tensors, one stream buffer each (at capacity) and outputs."""
+    raw: List[torch.Tensor]
+    streams: List[torch.Tensor] = field(default_factory=list)
+    outs: List[torch.Tensor] = field(default_factory=list)
+    sizes: Optional[torch.Tensor] = None      # int64 [n]: stream lengths, written by the device
+    status: Optional[torch.Tensor] = None     # int32 [1]: first device error of any call
+
+    @classmethod
+    def allocate(cls, raw: List[torch.Tensor], share_output: bool = False) -> "CodecSet":
+        dev = raw[0].device
+        cs = cls(raw=[t.contiguous() for t in raw])
+        cs.streams = [torch.empty(enec.enec_max_compressed_size(_DT[t.dtype], t.numel()), dtype=torch.uint8, device=dev)
+                      for t in cs.raw]
+        if share_output:
+            biggest = max(t.numel() for t in cs.raw)
+            pool = {dt: torch.empty(biggest, dtype=dt, device=dev) for dt in {t.dtype for t in cs.raw}}
+            cs.outs = [pool[t.dtype][:t.numel()] for t in cs.raw]
+        else:
+            cs.outs = [torch.empty(t.numel(), dtype=t.dtype, device=dev) for t in cs.raw]
+        cs.sizes = torch.zeros(len(cs.raw), dtype=torch.int64, device=dev)
+        cs.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        return cs
+
+    @property
+    def raw_bytes(self) -> int:
+        return sum(t.numel() * 2 for t in self.raw)
+
+    def compress_all(self, params=None) -> None:
+        """One enec_compress per tensor on the current stream (no host synchronisation)."""
+        for i, t in enumerate(self.raw):
+            dt = _DT[t.dtype]
+            if params is None:
+                st = enec.enec_compress(t, dt, t.numel(), self.streams[i], self.streams[i].numel(),
+                                        self.sizes[i:i + 1], self.status)
+            else:
+                st = enec.enec_compress_with_params(t, dt, t.numel(), *params, self.streams[i],
+                                                    self.streams[i].numel(), self.sizes[i:i + 1], self.status)
+            if st != 0:
+                raise enec.EnecError(st, f"enec_compress tensor {i}")
+
+    def decompress_all(self) -> None:
+        """One enec_decompress per tensor on the current stream. The stream length passed is the buffer's
+        capacity; the true length is in the stream header and is checked against it on the device."""
+        for i, t in enumerate(self.raw):
+            st = enec.enec_decompress(self.streams[i], self.streams[i].numel(), _DT[t.dtype], t.numel(),
+                                      self.outs[i], self.status)
+            if st != 0:
+                raise enec.EnecError(st, f"enec_decompress tensor {i}")
+
+    def check_status(self) -> None:
+        code = int(self.status.item())
+        if code != 0:
+            raise enec.EnecError(code, "device status")
+
+    def compressed_bytes(self) -> int:
+        return int(self.sizes.sum().item())
+
+    def verify_roundtrip(self) -> None:
+        """Outputs must equal the raw tensors bit for bit (needs unshared outputs)."""
+        for i, t in enumerate(self.raw):
+            if not torch.equal(self.outs[i].view(torch.int16), t.reshape(-1).view(torch.int16)):
+                raise AssertionError(f"tensor {i}: decompressed bits differ from the input")
