@@ -1,11 +1,14 @@
 // Decompression kernel: unpack + reconstruct (Sec. 5.1 decompression flow).
 //
-// One persistent CTA per resident slot. A producer warp stages each 16384-element block's compressed
+// One persistent CTA per resident slot. A loader warp stages each 16384-element block's compressed
 // segments (group mask, low plane, fp16 sign/mantissa-high plane, sign/mantissa bytes, wide-group
-// records) into shared memory with bulk asynchronous copies completing on an mbarrier; eight consumer
-// warps undo Algorithm 2 on packed bytes (four elements per 32-bit operation), locate each wide group's
-// record with a popcount prefix over the block's mask, apply the inverse transform of Sec. 5.3 and
-// write 16-byte coalesced stores. Every wait is bounded and ends in an error status, never a hang.
+// records) into shared memory with bulk asynchronous copies completing on an mbarrier. Eight consumer
+// warps first turn the block's mask into per-group record ranks (popcount prefix) and expand the staged
+// records to one byte per value, meet at a named barrier, then undo Algorithm 2 on packed bytes (four
+// elements per 32-bit operation), merge the high bits of wide groups, apply the inverse transform of
+// Sec. 5.3 and write 16-byte coalesced stores. Full blocks whose records all fit in the stage take a
+// branch-free body; tail blocks and overfull blocks take a general one. Every wait is bounded and ends
+// in an error status, never a hang.
 #pragma once
 
 #include "enec_common.cuh"
@@ -206,7 +209,8 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
 // Shared-memory layout of one pipeline stage (offsets from the stage base; all multiples of 16).
 //   meta | mask | rank array | low plane | fp16 sm-hi plane | sm bytes | raw records | expanded records
 // rank array: one u16 per group = rank of the group's record inside the block, or kNotWide.
-// expanded records: sixteen bytes per wide group (its high bits, one element per byte), rank order.
+// expanded records: sixteen bytes per wide group (its high bits, one element per byte), rank order, and
+// one all-zero slot at index cap that the rank entries of narrow groups point to in blocks that fit.
 // cap = records per block that fit; records beyond it are read from global memory by the consumers.
 struct StageLayout {
     uint32_t mask, rank, low, smhi, sm, raw, expanded, cap, bytes;
@@ -221,13 +225,13 @@ __device__ __forceinline__ StageLayout make_stage_layout(int dt, int m, int hbit
     L.raw = L.sm + kBlockElems;
     nstages = 2;
     uint32_t per_stage = (budget / 2) & ~15u;
-    if (per_stage < L.raw + 48) { nstages = 1; per_stage = budget & ~15u; }
-    if (per_stage < L.raw + 48) { nstages = 0; per_stage = L.raw + 48; }
-    uint32_t cap = hbits > 0 ? (per_stage - L.raw - 48) / uint32_t(2 * hbits + 16) : 0;
+    if (per_stage < L.raw + 64) { nstages = 1; per_stage = budget & ~15u; }
+    if (per_stage < L.raw + 64) { nstages = 0; per_stage = L.raw + 64; }
+    uint32_t cap = hbits > 0 ? (per_stage - L.raw - 64) / uint32_t(2 * hbits + 16) : 0;
     if (cap > kGroupsPerBlock) cap = kGroupsPerBlock;
     L.cap = cap;
     L.expanded = L.raw + uint32_t(align16(uint64_t(cap) * 2 * hbits + 32));
-    L.bytes = L.expanded + cap * 16;
+    L.bytes = L.expanded + (cap + 1) * 16;
     if (nstages == 2) {
         int more = int(budget / L.bytes);
         nstages = more > kMaxStages ? kMaxStages : more;
@@ -352,20 +356,69 @@ __device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, ui
     }
 }
 
-// Loader/expander warp, one block: per-group ranks from the mask, then the block's first `cap` records
-// expanded to sixteen bytes each. All 32 lanes.
-template <int HB>
-__device__ __forceinline__ void expand_records(uint32_t s_raw, uint32_t s_expanded, uint32_t count, uint32_t lane) {
-    for (uint32_t i = lane; i < count; i += 32) {
-        const uint32_t rp = s_raw + i * (2 * HB);
-        const uint4 v = unpack_record<HB>([&](int w) { return lds16(rp + 2 * w); });
-        sts128(s_expanded + i * 16, v);
+// Branch-free body for a full block (16384 real elements) whose records are all expanded in shared memory:
+// the rank entry of a narrow group points to the all-zero slot, so every run merges "its" high bits.
+// tid = 0..255; thread tid owns the runs c * 2048 + 8 tid (c < 8).
+template <int DT, int M, int HB>
+__device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_low, uint32_t s_smhi, uint32_t tid) {
+    constexpr int n = M + HB;
+    constexpr uint32_t Hm = 0x80808080u;
+    uint2 y[8];
+    uint2 hs[8];
+    unpack_plane<M>(s_low, 8 * tid, kBlockElems, y);
+    if (DT == ENEC_FP16) unpack_plane<3>(s_smhi, 8 * tid, kBlockElems, hs);
+    const uint32_t rank_addr = r.rank + (tid >> 1) * 2;
+    const uint32_t exp_addr = r.expanded + (tid & 1) * 8;
+    const uint32_t sm_addr = r.sm + 8 * tid;
+    uint4* out = reinterpret_cast<uint4*>(r.out + 8 * tid);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint2 v = y[c];
+        if constexpr (HB > 0) {
+            const uint32_t rk = lds16(rank_addr + c * (kBlockElems / 8 / 16) * 2);
+            const uint2 hi = lds64(exp_addr + rk * 16);
+            v.x += hi.x << M;  // disjoint bits
+            v.y += hi.y << M;
+        }
+        uint32_t x0, x1;
+        if constexpr (n < 8) {
+            x0 = (r.c4_or_h - (v.x ^ r.s4)) ^ r.fix;
+            x1 = (r.c4_or_h - (v.y ^ r.s4)) ^ r.fix;
+        } else {
+            x0 = ((r.b4 | Hm) - (v.x & ~Hm)) ^ ((r.b4 ^ ~v.x) & Hm);
+            x1 = ((r.b4 | Hm) - (v.y & ~Hm)) ^ ((r.b4 ^ ~v.y) & Hm);
+        }
+        const uint2 smv = lds64(sm_addr + c * (kBlockElems / 8));
+        uint32_t lo0, lo1, hi0, hi1;
+        if (DT == ENEC_BF16) {
+            hi0 = (smv.x & Hm) | ((x0 >> 1) & ~Hm);
+            hi1 = (smv.y & Hm) | ((x1 >> 1) & ~Hm);
+            lo0 = ((x0 << 7) & Hm) | (smv.x & ~Hm);
+            lo1 = ((x1 << 7) & Hm) | (smv.y & ~Hm);
+        } else {
+            x0 &= 0x1F1F1F1Fu;
+            x1 &= 0x1F1F1F1Fu;
+            hi0 = ((hs[c].x << 5) & Hm) | (x0 << 2) | (hs[c].x & 0x03030303u);
+            hi1 = ((hs[c].y << 5) & Hm) | (x1 << 2) | (hs[c].y & 0x03030303u);
+            lo0 = smv.x;
+            lo1 = smv.y;
+        }
+        uint4 w;
+        w.x = prmt(lo0, hi0, 0x5140u);
+        w.y = prmt(lo0, hi0, 0x7362u);
+        w.z = prmt(lo1, hi1, 0x5140u);
+        w.w = prmt(lo1, hi1, 0x7362u);
+        out[c * (kBlockElems / 8 / 8)] = w;
     }
 }
 
-__device__ __forceinline__ uint32_t build_rank_array(uint32_t s_mask, uint32_t s_rank, uint32_t N, uint32_t lane) {
+// Consumer preparation of a block, all 256 consumer threads: per-group record ranks from the mask
+// (popcount prefix; a narrow group gets `narrow_entry`). Returns the number of wide groups the mask holds.
+__device__ __forceinline__ uint32_t build_rank_array(uint32_t s_mask, uint32_t s_rank, uint32_t N, uint32_t tid,
+                                                     uint32_t narrow_entry) {
+    const uint32_t lane = tid & 31;
     const uint32_t groups = N >> 4;
-    uint32_t mw = 0;
+    uint32_t mw = 0;  // every warp holds all 32 mask words, one per lane
     if (lane * 32 < groups) {
         mw = lds32(s_mask + 4 * lane);
         if (groups - lane * 32 < 32) mw &= (1u << (groups - lane * 32)) - 1;
@@ -376,26 +429,66 @@ __device__ __forceinline__ uint32_t build_rank_array(uint32_t s_mask, uint32_t s
         const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
         if (lane >= uint32_t(d)) incl += t;
     }
-    uint32_t run = incl - __popc(mw);
-    if (lane * 32 < groups) {
-#pragma unroll
-        for (int b = 0; b < 32; b += 2) {
-            const uint32_t r0 = (mw >> b) & 1 ? run : kNotWide;
-            run += (mw >> b) & 1;
-            const uint32_t r1 = (mw >> (b + 1)) & 1 ? run : kNotWide;
-            run += (mw >> (b + 1)) & 1;
-            sts32(s_rank + (lane * 32 + b) * 2, r0 | (r1 << 16));
-        }
+    // thread tid writes the entries of groups 4 tid .. 4 tid + 3 (word tid / 8, bits 4 (tid % 8) ..)
+    const uint32_t word = tid >> 3, bit0 = (tid & 7) * 4;
+    const uint32_t w = __shfl_sync(0xFFFFFFFFu, mw, word);
+    uint32_t run = __shfl_sync(0xFFFFFFFFu, incl - __popc(mw), word) + __popc(w & ((1u << bit0) - 1));
+    const uint32_t bits = (w >> bit0) & 15;
+    const uint32_t e0 = bits & 1 ? run : narrow_entry;
+    run += bits & 1;
+    const uint32_t e1 = bits & 2 ? run : narrow_entry;
+    run += (bits >> 1) & 1;
+    const uint32_t e2 = bits & 4 ? run : narrow_entry;
+    run += (bits >> 2) & 1;
+    const uint32_t e3 = bits & 8 ? run : narrow_entry;
+    if (4 * tid < groups) sts64(s_rank + 8 * tid, make_uint2(e0 | (e1 << 16), e2 | (e3 << 16)));
+    return __shfl_sync(0xFFFFFFFFu, incl, 31);
+}
+
+// The staged records expanded to sixteen bytes each (one value per byte), all consumer threads.
+template <int HB>
+__device__ __forceinline__ void expand_records(uint32_t s_raw, uint32_t s_expanded, uint32_t count, uint32_t tid) {
+    for (uint32_t i = tid; i < count; i += kConsumerWarps * 32) {
+        const uint32_t rp = s_raw + i * (2 * HB);
+        const uint4 v = unpack_record<HB>([&](int w) { return lds16(rp + 2 * w); });
+        sts128(s_expanded + i * 16, v);
     }
-    return __shfl_sync(0xFFFFFFFFu, incl, 31);  // wide groups in the block according to the mask
+}
+
+__device__ __forceinline__ void expand_records_any(int hbits, uint32_t s_raw, uint32_t s_expanded, uint32_t count,
+                                                   uint32_t tid) {
+    switch (hbits) {
+        case 0: break;
+        case 1: expand_records<1>(s_raw, s_expanded, count, tid); break;
+        case 2: expand_records<2>(s_raw, s_expanded, count, tid); break;
+        case 3: expand_records<3>(s_raw, s_expanded, count, tid); break;
+        case 4: expand_records<4>(s_raw, s_expanded, count, tid); break;
+        case 5: expand_records<5>(s_raw, s_expanded, count, tid); break;
+        case 6: expand_records<6>(s_raw, s_expanded, count, tid); break;
+        default: expand_records<7>(s_raw, s_expanded, count, tid); break;
+    }
+}
+
+// Barrier of the consumer threads only (the loader warp does not take part) that also ORs a flag over
+// them, so that all consumers take the same decision whatever the moment another warp raised the flag.
+__device__ __forceinline__ bool consumer_barrier_or(bool flag) {
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(any)
+        : "r"(uint32_t(flag)), "n"(kConsumerWarps * 32)
+        : "memory");
+    return any != 0;
 }
 
 struct DecodeShared {
     uint64_t full[kMaxStages];   // bulk copies of a stage have landed
-    uint64_t ready[kMaxStages];  // rank array and expanded records of a stage are written
     uint64_t empty[kMaxStages];  // all consumer warps are done with a stage
     int abort;
-    int pad[7];
+    int pad[15];
 };
 static_assert(sizeof(DecodeShared) == 128, "control area is 128 bytes");
 
@@ -453,12 +546,13 @@ enec_decode_kernel(DecodeJob job, int* status) {
     if (threadIdx.x == 0) {
         for (int s = 0; s < nstages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->ready[s], 1);
             mbar_init(&ctl->empty[s], kConsumerWarps);
         }
         ctl->abort = 0;
         mbar_fence_init();
     }
+    if (threadIdx.x < uint32_t(nstages))  // the all-zero record slot of every stage
+        sts128(stages + threadIdx.x * L.bytes + L.expanded + L.cap * 16, make_uint4(0, 0, 0, 0));
     __syncthreads();
 
     const uint32_t warp = threadIdx.x >> 5;
@@ -466,104 +560,64 @@ enec_decode_kernel(DecodeJob job, int* status) {
     volatile int* abort_flag = &ctl->abort;
     const uint32_t n_mine = jc.nblocks > blockIdx.x ? (jc.nblocks - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const uint32_t S = uint32_t(nstages);
+    const uint32_t* table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
 
     if (warp == kConsumerWarps) {
-        // ---------------- loader + expander warp ----------------
-        const uint32_t* table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
-        uint32_t next_load = 0, next_exp = 0;
-        uint32_t t0 = 0, t1 = 0;  // table entries of block next_load (lane 0)
-        if (lane == 0 && n_mine) { t0 = table[blockIdx.x]; t1 = table[blockIdx.x + 1]; }
+        // ---------------- loader warp: lane 0 issues the copies of block after block ----------------
+        if (lane != 0) return;
+        uint32_t issued = 0;
         bool failed = false;
-        while (next_exp < n_mine && !failed) {
-            // issue every load that has a free stage; block only when there is nothing to expand
-            while (next_load < n_mine && next_load < next_exp + S) {
-                const uint32_t s = next_load % S, use = next_load / S;
-                if (use > 0) {
-                    bool free_now;
-                    if (next_exp < next_load) {
-                        int f = lane == 0 ? int(mbar_try_wait(&ctl->empty[s], (use - 1) & 1)) : 0;
-                        free_now = __shfl_sync(0xFFFFFFFFu, f, 0) != 0;
-                        if (!free_now) break;
-                    } else if (!warp_wait(&ctl->empty[s], (use - 1) & 1, abort_flag, lane)) {
-                        failed = true;
-                        break;
-                    }
+        for (; issued < n_mine; ++issued) {
+            const uint32_t s = issued % S, use = issued / S;
+            if (use > 0) {
+                bool freed = false;
+                for (uint32_t it = 0; it < (1u << 22); ++it) {
+                    if (mbar_try_wait(&ctl->empty[s], (use - 1) & 1)) { freed = true; break; }
+                    if (*abort_flag) break;
+                    if (it > 16) __nanosleep(64);
                 }
-                int bad = 0;
-                if (lane == 0) {
-                    const uint32_t k = blockIdx.x + next_load * gridDim.x;
-                    const bool tail = (k + 1 == jc.nblocks);
-                    const uint32_t N = tail ? jc.tail_padded : kBlockElems;
-                    const uint32_t real = tail ? jc.tail_real : kBlockElems;
-                    const uint64_t h0 = jc.off_high + uint64_t(t0) * (2 * hbits);
-                    const uint64_t w0 = h0 & ~uint64_t(15);
-                    bad = t1 < t0 || t1 - t0 > (N >> 4) || t1 > jc.a_total;
-                    if (!bad) {
-                        uint32_t staged = t1 - t0 < L.cap ? t1 - t0 : L.cap;   // records staged and expanded
-                        if (hbits == 0) staged = 0;
-                        const uint64_t w1 = align16(h0 + uint64_t(staged) * (2 * hbits));
-                        const uint32_t mask_bytes = uint32_t(align16(((N >> 4) + 7) / 8));
-                        const uint32_t low_bytes = uint32_t(align16(uint64_t(N) * jc.m / 8));
-                        const uint32_t smhi_bytes = DT == ENEC_FP16 ? uint32_t(align16(uint64_t(N) * 3 / 8)) : 0;
-                        const uint32_t sm_bytes = uint32_t(align16(real));
-                        const uint32_t raw_bytes = staged ? uint32_t(w1 - w0) : 0;
-                        uint8_t* st = smem + sizeof(DecodeShared) + size_t(s) * L.bytes;
-                        uint32_t* meta = reinterpret_cast<uint32_t*>(st);
-                        meta[0] = uint32_t(h0 - w0);  // offset of the first record inside the staged window
-                        meta[1] = staged;
-                        meta[2] = t1 - t0;
-                        mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes);
-                        bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
-                        bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
-                        if (DT == ENEC_FP16)
-                            bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
-                        bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
-                        if (raw_bytes) bulk_g2s(st + L.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
-                        if (next_load + 1 < n_mine) { t0 = table[k + gridDim.x]; t1 = table[k + gridDim.x + 1]; }
-                    }
-                }
-                if (__shfl_sync(0xFFFFFFFFu, bad, 0)) {
-                    if (lane == 0) { *abort_flag = 1; report(status, ENEC_ERR_BAD_STREAM); }
-                    failed = true;
-                    break;
-                }
-                ++next_load;
+                if (!freed) { failed = true; break; }
             }
-            if (failed || next_exp >= next_load) continue;
-            // expand the oldest loaded block
-            const uint32_t s = next_exp % S, use = next_exp / S;
-            if (!warp_wait(&ctl->full[s], use & 1, abort_flag, lane)) { failed = true; break; }
-            const uint32_t k = blockIdx.x + next_exp * gridDim.x;
-            const uint32_t N = (k + 1 == jc.nblocks) ? jc.tail_padded : kBlockElems;
-            const uint32_t st = stages + s * L.bytes;
-            const uint32_t first = lds32(st), staged = lds32(st + 4), expect = lds32(st + 8);
-            if (hbits > 0) {
-                const uint32_t wide = build_rank_array(st + L.mask, st + L.rank, N, lane);
-                if (wide != expect) {  // the prefix table must agree with the mask
-                    if (lane == 0) { *abort_flag = 1; report(status, ENEC_ERR_BAD_STREAM); }
-                    failed = true;
-                    break;
-                }
-                switch (hbits) {
-                    case 1: expand_records<1>(st + L.raw + first, st + L.expanded, staged, lane); break;
-                    case 2: expand_records<2>(st + L.raw + first, st + L.expanded, staged, lane); break;
-                    case 3: expand_records<3>(st + L.raw + first, st + L.expanded, staged, lane); break;
-                    case 4: expand_records<4>(st + L.raw + first, st + L.expanded, staged, lane); break;
-                    case 5: expand_records<5>(st + L.raw + first, st + L.expanded, staged, lane); break;
-                    case 6: expand_records<6>(st + L.raw + first, st + L.expanded, staged, lane); break;
-                    default: expand_records<7>(st + L.raw + first, st + L.expanded, staged, lane); break;
-                }
+            const uint32_t k = blockIdx.x + issued * gridDim.x;
+            const bool tail = (k + 1 == jc.nblocks);
+            const uint32_t N = tail ? jc.tail_padded : kBlockElems;
+            const uint32_t real = tail ? jc.tail_real : kBlockElems;
+            const uint32_t t0 = table[k], t1 = table[k + 1];
+            if (t1 < t0 || t1 - t0 > (N >> 4) || t1 > jc.a_total) {
+                *abort_flag = 1;
+                report(status, ENEC_ERR_BAD_STREAM);
+                failed = true;
+                break;
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->ready[s]);
-            ++next_exp;
+            const uint64_t h0 = jc.off_high + uint64_t(t0) * (2 * hbits);
+            const uint64_t w0 = h0 & ~uint64_t(15);
+            uint32_t staged = t1 - t0 < L.cap ? t1 - t0 : L.cap;  // records staged in shared memory
+            if (hbits == 0) staged = 0;
+            const uint64_t w1 = align16(h0 + uint64_t(staged) * (2 * hbits));
+            const uint32_t mask_bytes = uint32_t(align16(((N >> 4) + 7) / 8));
+            const uint32_t low_bytes = uint32_t(align16(uint64_t(N) * jc.m / 8));
+            const uint32_t smhi_bytes = DT == ENEC_FP16 ? uint32_t(align16(uint64_t(N) * 3 / 8)) : 0;
+            const uint32_t sm_bytes = uint32_t(align16(real));
+            const uint32_t raw_bytes = staged ? uint32_t(w1 - w0) : 0;
+            uint8_t* st = smem + sizeof(DecodeShared) + size_t(s) * L.bytes;
+            uint32_t* meta = reinterpret_cast<uint32_t*>(st);
+            meta[0] = uint32_t(h0 - w0);  // offset of the first record inside the staged window
+            meta[1] = staged;
+            meta[2] = t1 - t0;
+            meta[3] = t0;
+            mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes);
+            bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
+            bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
+            if (DT == ENEC_FP16)
+                bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
+            bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
+            if (raw_bytes) bulk_g2s(st + L.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
         }
         if (failed) {
-            if (lane == 0) {
-                if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
-                // let copies still in flight land before the CTA's shared memory is released
-                for (uint32_t i = next_exp; i < next_load; ++i) mbar_wait_bounded(&ctl->full[i % S], (i / S) & 1);
-            }
+            if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
+            // let copies still in flight land before the CTA's shared memory is released
+            const uint32_t from = issued > S ? issued - S : 0;
+            for (uint32_t i = from; i < issued; ++i) mbar_wait_bounded(&ctl->full[i % S], (i / S) & 1);
         }
         return;
     }
@@ -581,33 +635,57 @@ enec_decode_kernel(DecodeJob job, int* status) {
         r.cap = L.cap;
     }
     const int code = jc.m * 8 + hbits;
+    const uint32_t tid = threadIdx.x;
     for (uint32_t i = 0; i < n_mine; ++i) {
         const uint32_t s = i % S, use = i / S;
-        if (!warp_wait(&ctl->ready[s], use & 1, abort_flag, lane)) {
-            if (lane == 0 && !*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
-            break;
-        }
-        mbar_try_wait(&ctl->full[s], use & 1);  // the staged bytes themselves (already complete)
         const uint32_t k = blockIdx.x + i * gridDim.x;
         const bool tail = (k + 1 == jc.nblocks);
         const uint32_t N = tail ? jc.tail_padded : kBlockElems;
         const uint32_t st = stages + s * L.bytes;
+        bool fits = false;
+        bool failed = false;
+        if (warp_wait(&ctl->full[s], use & 1, abort_flag, lane)) {
+            // preparation: ranks of the wide groups and expanded records
+            const uint32_t first = lds32(st), staged = lds32(st + 4), expect = lds32(st + 8);
+            fits = expect <= L.cap;
+            if (hbits > 0) {
+                // the branch-free body (full blocks that fit) wants narrow groups to point at the zero slot
+                const uint32_t wide = build_rank_array(st + L.mask, st + L.rank, N, tid, fits && !tail ? L.cap : kNotWide);
+                if (wide != expect) {  // the prefix table must agree with the mask
+                    if (lane == 0) { *abort_flag = 1; report(status, ENEC_ERR_BAD_STREAM); }
+                }
+                expand_records_any(hbits, st + L.raw + first, st + L.expanded, staged, tid);
+            }
+            r.high = jc.in + jc.off_high + uint64_t(lds32(st + 12)) * (2 * hbits);
+        } else {
+            failed = true;
+            if (lane == 0 && !*abort_flag) {
+                *abort_flag = 1;
+                report(status, ENEC_ERR_TIMEOUT);
+            }
+        }
+        // every consumer warp reaches this once per block, failed wait or not, and all leave together
+        if (consumer_barrier_or(failed || *abort_flag != 0)) break;
         r.sm = st + L.sm;
         r.rank = st + L.rank;
         r.expanded = st + L.expanded;
-        r.high = jc.in + jc.off_high + uint64_t(reinterpret_cast<const uint32_t*>(jc.in + jc.off_table)[k]) * (2 * hbits);
         r.out = jc.out + uint64_t(k) * kBlockElems;
         r.real = tail ? jc.tail_real : kBlockElems;
+        const bool full_block = !tail && fits;
         switch (code) {
-#define ENEC_CASE(DTV, MV, HV)                                                        \
-    case MV * 8 + HV:                                                                 \
-        decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, threadIdx.x);        \
+#define ENEC_CASE(DTV, MV, HV)                                                               \
+    case MV * 8 + HV:                                                                        \
+        if (full_block) decode_full_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, tid);     \
+        else decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, tid);                  \
         break;
             ENEC_FOR_EACH_MH(ENEC_CASE, DT)
 #undef ENEC_CASE
-#define ENEC_CASE(DTV, MV, HV)                                                        \
-    case MV * 8 + HV:                                                                 \
-        if constexpr (DTV == ENEC_BF16) decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, threadIdx.x); \
+#define ENEC_CASE(DTV, MV, HV)                                                               \
+    case MV * 8 + HV:                                                                        \
+        if constexpr (DTV == ENEC_BF16) {                                                    \
+            if (full_block) decode_full_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, tid); \
+            else decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, tid);              \
+        }                                                                                    \
         break;
             ENEC_FOR_EACH_MH_BF16_ONLY(ENEC_CASE, DT)
 #undef ENEC_CASE
