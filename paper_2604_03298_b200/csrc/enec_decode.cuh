@@ -248,6 +248,7 @@ struct RunCtx {
     uint16_t* out;        // global: first element of the block
     uint32_t real;        // real elements in the block
     uint32_t c4_or_h, fix, s4, b4;  // packed transform constants
+    uint32_t c4;                    // rep4(b + 2^(n-1)) when that sum fits a byte
     int n;
 };
 
@@ -356,8 +357,12 @@ __device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, ui
     }
 }
 
-// Branch-free body for a full block (16384 real elements) whose records are all expanded in shared memory:
-// the rank entry of a narrow group points to the all-zero slot, so every run merges "its" high bits.
+// Branch-free body for a full block (16384 real elements) whose records are all expanded in shared memory.
+// The expanded high bits are stored with the sign position 2^(n-1) already flipped, and the rank entry of
+// a narrow group points to a slot that holds just that flip, so low + (slot << M) is y ^ 2^(n-1) for every
+// run. bf16 with n < 8 uses it only when b + 2^(n-1) <= 255: then x = (b + 2^(n-1)) - (y ^ 2^(n-1)) never
+// borrows across bytes for a stream that came from real data (x is a field value), and a plain
+// subtraction serves; other bf16 tensors with n < 8 take the general body.
 // tid = 0..255; thread tid owns the runs c * 2048 + 8 tid (c < 8).
 template <int DT, int M, int HB>
 __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_low, uint32_t s_smhi, uint32_t tid) {
@@ -379,14 +384,21 @@ __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_lo
             const uint2 hi = lds64(exp_addr + rk * 16);
             v.x += hi.x << M;  // disjoint bits
             v.y += hi.y << M;
+        } else {
+            v.x ^= r.s4;
+            v.y ^= r.s4;
         }
         uint32_t x0, x1;
-        if constexpr (n < 8) {
-            x0 = (r.c4_or_h - (v.x ^ r.s4)) ^ r.fix;
-            x1 = (r.c4_or_h - (v.y ^ r.s4)) ^ r.fix;
-        } else {
-            x0 = ((r.b4 | Hm) - (v.x & ~Hm)) ^ ((r.b4 ^ ~v.x) & Hm);
-            x1 = ((r.b4 | Hm) - (v.y & ~Hm)) ^ ((r.b4 ^ ~v.y) & Hm);
+        if constexpr (DT == ENEC_FP16) {
+            // b + 2^(n-1) < 128: the guard bit absorbs any borrow and is masked away with the field
+            x0 = r.c4_or_h - v.x;
+            x1 = r.c4_or_h - v.y;
+        } else if constexpr (n < 8) {
+            x0 = r.c4 - v.x;
+            x1 = r.c4 - v.y;
+        } else {  // n = 8: bytewise (b + 128) - (y ^ 128) modulo 256
+            x0 = (r.c4_or_h - (v.x & ~Hm)) ^ ((r.c4 ^ ~v.x) & Hm);
+            x1 = (r.c4_or_h - (v.y & ~Hm)) ^ ((r.c4 ^ ~v.y) & Hm);
         }
         const uint2 smv = lds64(sm_addr + c * (kBlockElems / 8));
         uint32_t lo0, lo1, hi0, hi1;
@@ -446,26 +458,29 @@ __device__ __forceinline__ uint32_t build_rank_array(uint32_t s_mask, uint32_t s
 }
 
 // The staged records expanded to sixteen bytes each (one value per byte), all consumer threads.
+// `flip` is XORed into every expanded word (the branch-free body wants the sign position flipped).
 template <int HB>
-__device__ __forceinline__ void expand_records(uint32_t s_raw, uint32_t s_expanded, uint32_t count, uint32_t tid) {
+__device__ __forceinline__ void expand_records(uint32_t s_raw, uint32_t s_expanded, uint32_t count, uint32_t tid,
+                                               uint32_t flip) {
     for (uint32_t i = tid; i < count; i += kConsumerWarps * 32) {
         const uint32_t rp = s_raw + i * (2 * HB);
-        const uint4 v = unpack_record<HB>([&](int w) { return lds16(rp + 2 * w); });
+        uint4 v = unpack_record<HB>([&](int w) { return lds16(rp + 2 * w); });
+        v.x ^= flip; v.y ^= flip; v.z ^= flip; v.w ^= flip;
         sts128(s_expanded + i * 16, v);
     }
 }
 
 __device__ __forceinline__ void expand_records_any(int hbits, uint32_t s_raw, uint32_t s_expanded, uint32_t count,
-                                                   uint32_t tid) {
+                                                   uint32_t tid, uint32_t flip) {
     switch (hbits) {
         case 0: break;
-        case 1: expand_records<1>(s_raw, s_expanded, count, tid); break;
-        case 2: expand_records<2>(s_raw, s_expanded, count, tid); break;
-        case 3: expand_records<3>(s_raw, s_expanded, count, tid); break;
-        case 4: expand_records<4>(s_raw, s_expanded, count, tid); break;
-        case 5: expand_records<5>(s_raw, s_expanded, count, tid); break;
-        case 6: expand_records<6>(s_raw, s_expanded, count, tid); break;
-        default: expand_records<7>(s_raw, s_expanded, count, tid); break;
+        case 1: expand_records<1>(s_raw, s_expanded, count, tid, flip); break;
+        case 2: expand_records<2>(s_raw, s_expanded, count, tid, flip); break;
+        case 3: expand_records<3>(s_raw, s_expanded, count, tid, flip); break;
+        case 4: expand_records<4>(s_raw, s_expanded, count, tid, flip); break;
+        case 5: expand_records<5>(s_raw, s_expanded, count, tid, flip); break;
+        case 6: expand_records<6>(s_raw, s_expanded, count, tid, flip); break;
+        default: expand_records<7>(s_raw, s_expanded, count, tid, flip); break;
     }
 }
 
@@ -508,19 +523,15 @@ static_assert(sizeof(DecodeShared) == 128, "control area is 128 bytes");
     X(DT, 7, 0) X(DT, 7, 1)                                                                           \
     X(DT, 8, 0)
 
-// Bounded wait by lane 0 with the result broadcast to the warp; also gives up when the CTA aborts.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t lane) {
-    int ok = 0;
-    if (lane == 0) {
-        for (uint32_t it = 0; it < (1u << 22); ++it) {
-            if (mbar_try_wait(bar, parity)) { ok = 1; break; }
-            if (*abort_flag) break;
-            if (it > 16) __nanosleep(64);
-        }
+// Bounded wait by one thread; also gives up when the CTA aborts. Sleeps between polls so that a waiting
+// thread leaves the issue slots to the warps that have work.
+__device__ __forceinline__ bool poll_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        __nanosleep(it < 64 ? 32 : 256);
     }
-    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-    if (ok && lane != 0) mbar_try_wait(bar, parity);  // acquire in every lane
-    return ok != 0;
+    return false;
 }
 
 template <int DT>
@@ -551,8 +562,10 @@ enec_decode_kernel(DecodeJob job, int* status) {
         ctl->abort = 0;
         mbar_fence_init();
     }
-    if (threadIdx.x < uint32_t(nstages))  // the all-zero record slot of every stage
-        sts128(stages + threadIdx.x * L.bytes + L.expanded + L.cap * 16, make_uint4(0, 0, 0, 0));
+    // the slot narrow groups point to in the branch-free body: no high bits, sign position flipped
+    const uint32_t flip4 = hbits > 0 ? rep4(1u << (hbits - 1)) : 0;
+    if (threadIdx.x < uint32_t(nstages))
+        sts128(stages + threadIdx.x * L.bytes + L.expanded + L.cap * 16, make_uint4(flip4, flip4, flip4, flip4));
     __syncthreads();
 
     const uint32_t warp = threadIdx.x >> 5;
@@ -567,22 +580,15 @@ enec_decode_kernel(DecodeJob job, int* status) {
         if (lane != 0) return;
         uint32_t issued = 0;
         bool failed = false;
+        uint32_t t0 = 0, t1 = 0;  // table entries of the next block to issue, fetched one block ahead
+        if (n_mine) { t0 = table[blockIdx.x]; t1 = table[blockIdx.x + 1]; }
         for (; issued < n_mine; ++issued) {
             const uint32_t s = issued % S, use = issued / S;
-            if (use > 0) {
-                bool freed = false;
-                for (uint32_t it = 0; it < (1u << 22); ++it) {
-                    if (mbar_try_wait(&ctl->empty[s], (use - 1) & 1)) { freed = true; break; }
-                    if (*abort_flag) break;
-                    if (it > 16) __nanosleep(64);
-                }
-                if (!freed) { failed = true; break; }
-            }
+            if (use > 0 && !poll_wait(&ctl->empty[s], (use - 1) & 1, abort_flag)) { failed = true; break; }
             const uint32_t k = blockIdx.x + issued * gridDim.x;
             const bool tail = (k + 1 == jc.nblocks);
             const uint32_t N = tail ? jc.tail_padded : kBlockElems;
             const uint32_t real = tail ? jc.tail_real : kBlockElems;
-            const uint32_t t0 = table[k], t1 = table[k + 1];
             if (t1 < t0 || t1 - t0 > (N >> 4) || t1 > jc.a_total) {
                 *abort_flag = 1;
                 report(status, ENEC_ERR_BAD_STREAM);
@@ -612,6 +618,7 @@ enec_decode_kernel(DecodeJob job, int* status) {
                 bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
             bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
             if (raw_bytes) bulk_g2s(st + L.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
+            if (issued + 1 < n_mine) { t0 = table[k + gridDim.x]; t1 = table[k + gridDim.x + 1]; }
         }
         if (failed) {
             if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
@@ -631,6 +638,7 @@ enec_decode_kernel(DecodeJob job, int* status) {
         r.c4_or_h = rep4(c) | 0x80808080u;
         r.fix = ~rep4(c) & 0x80808080u;
         r.b4 = rep4(uint32_t(jc.b));
+        r.c4 = rep4(c);
         r.n = jc.n;
         r.cap = L.cap;
     }
@@ -642,36 +650,35 @@ enec_decode_kernel(DecodeJob job, int* status) {
         const bool tail = (k + 1 == jc.nblocks);
         const uint32_t N = tail ? jc.tail_padded : kBlockElems;
         const uint32_t st = stages + s * L.bytes;
-        bool fits = false;
+        // one thread waits for the block's bytes; the others sleep at the barrier
         bool failed = false;
-        if (warp_wait(&ctl->full[s], use & 1, abort_flag, lane)) {
-            // preparation: ranks of the wide groups and expanded records
-            const uint32_t first = lds32(st), staged = lds32(st + 4), expect = lds32(st + 8);
-            fits = expect <= L.cap;
-            if (hbits > 0) {
-                // the branch-free body (full blocks that fit) wants narrow groups to point at the zero slot
-                const uint32_t wide = build_rank_array(st + L.mask, st + L.rank, N, tid, fits && !tail ? L.cap : kNotWide);
-                if (wide != expect) {  // the prefix table must agree with the mask
-                    if (lane == 0) { *abort_flag = 1; report(status, ENEC_ERR_BAD_STREAM); }
-                }
-                expand_records_any(hbits, st + L.raw + first, st + L.expanded, staged, tid);
-            }
-            r.high = jc.in + jc.off_high + uint64_t(lds32(st + 12)) * (2 * hbits);
-        } else {
+        if (tid == 0 && !poll_wait(&ctl->full[s], use & 1, abort_flag)) {
             failed = true;
-            if (lane == 0 && !*abort_flag) {
-                *abort_flag = 1;
-                report(status, ENEC_ERR_TIMEOUT);
-            }
+            if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
         }
-        // every consumer warp reaches this once per block, failed wait or not, and all leave together
+        // every consumer reaches both barriers of a block, failed wait or not, and all leave together
         if (consumer_barrier_or(failed || *abort_flag != 0)) break;
+        mbar_try_wait(&ctl->full[s], use & 1);  // completed: acquires the copied bytes in every thread
+        // preparation: ranks of the wide groups and expanded records
+        const uint32_t first = lds32(st), staged = lds32(st + 4), expect = lds32(st + 8);
+        const bool simple_sub = DT == ENEC_FP16 || jc.n == 8 || uint32_t(jc.b) + (1u << (jc.n - 1)) <= 255;
+        const bool full_block = !tail && expect <= L.cap && simple_sub;
+        if (hbits > 0) {
+            // the branch-free body wants narrow groups to point at the flip slot and flipped records
+            const uint32_t wide = build_rank_array(st + L.mask, st + L.rank, N, tid, full_block ? L.cap : kNotWide);
+            if (wide != expect && lane == 0) {  // the prefix table must agree with the mask
+                *abort_flag = 1;
+                report(status, ENEC_ERR_BAD_STREAM);
+            }
+            expand_records_any(hbits, st + L.raw + first, st + L.expanded, staged, tid, full_block ? flip4 : 0);
+        }
+        r.high = jc.in + jc.off_high + uint64_t(lds32(st + 12)) * (2 * hbits);
+        if (consumer_barrier_or(*abort_flag != 0)) break;
         r.sm = st + L.sm;
         r.rank = st + L.rank;
         r.expanded = st + L.expanded;
         r.out = jc.out + uint64_t(k) * kBlockElems;
         r.real = tail ? jc.tail_real : kBlockElems;
-        const bool full_block = !tail && fits;
         switch (code) {
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \

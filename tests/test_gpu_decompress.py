@@ -131,3 +131,29 @@ def test_host_argument_checks():
     assert enec.enec_decompress(buf[1:], 4000, 0, 64, out) == -1
     assert enec.enec_decompress(buf, 10, 0, 64, out) == -4
     assert enec.enec_decompress(None, 4096, 0, 64, out) == -1
+
+
+@pytest.mark.parametrize("b,n,m", [(250, 6, 3), (240, 5, 2), (3, 3, 1), (255, 8, 4), (200, 7, 7)])
+def test_exponents_near_the_ends_of_the_field(oracle, b, n, m):
+    # b + 2^(n-1) beyond 255 and b near 0: the byte arithmetic of the inverse transform must not leak between bytes
+    rng = np.random.default_rng(b)
+    count = 16384 * 6 + 100
+    half = 1 << (n - 1)
+    lo, hi = max(0, b - (half - 1)), min(255, b + half)
+    x = rng.integers(lo, hi + 1, count) if n < 8 else rng.integers(0, 256, count)
+    x = np.where(rng.random(count) < 0.7, np.clip(b - rng.integers(0, 1 << max(m - 1, 0), count), 0, 255), x)
+    words = ((x.astype(np.uint16) << 7) | rng.integers(0, 128, count).astype(np.uint16)
+             | (rng.integers(0, 2, count).astype(np.uint16) << 15)).astype(np.uint16)
+    check_roundtrip(oracle, words, 0, (b, n, m))
+
+
+def test_fp16_full_width_field(oracle):
+    # n = E = 5: b - y wraps modulo 32
+    rng = np.random.default_rng(77)
+    count = 16384 * 5 + 9
+    for b in (0, 7, 31):
+        x = rng.integers(0, 32, count)
+        words = ((x.astype(np.uint16) << 10) | rng.integers(0, 1024, count).astype(np.uint16)
+                 | (rng.integers(0, 2, count).astype(np.uint16) << 15)).astype(np.uint16)
+        for m in (1, 3, 5):
+            check_roundtrip(oracle, words, 1, (b, 5, m))
