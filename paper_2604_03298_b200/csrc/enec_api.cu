@@ -3,6 +3,7 @@
 #include <map>
 #include <mutex>
 #include <utility>
+#include <vector>
 
 #include "enec_decode.cuh"
 #include "enec_encode.cuh"
@@ -29,7 +30,7 @@ static DeviceInfo& device_info(int dev) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 template <int DT>
-static enec_status launch_decode(const DecodeJob& job, uint32_t nblocks, int* d_status, cudaStream_t stream) {
+static enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
     DeviceInfo& info = device_info(dev);
@@ -39,28 +40,29 @@ static enec_status launch_decode(const DecodeJob& job, uint32_t nblocks, int* d_
             return ENEC_ERR_CUDA;
         info.decode_attr_set[DT] = true;
     }
-    uint32_t grid = uint32_t(info.sms) * 3;
-    if (grid > nblocks) grid = nblocks;
+    uint32_t grid = uint32_t(info.sms) * 3;  // three resident CTAs per SM
+    if (grid > batch.total_blocks) grid = batch.total_blocks;
     if (grid == 0) grid = 1;
-    enec_decode_kernel<DT><<<grid, kDecodeThreads, kDecodeSmemBytes, stream>>>(job, d_status);
+    enec_decode_kernel<DT><<<grid, kDecodeThreads, kDecodeSmemBytes, stream>>>(batch, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
 
-
-// Device scratch of the compressor, one area per (device, stream): control words and one state word per
-// block. Grown when a larger tensor arrives; outgrown areas are kept until exit because work that uses
-// them may still be queued.
+// Device scratch, one area per (device, stream, purpose): for the compressor control words and one state
+// word per block, for a batched call the tensor descriptors. Grown when a larger request arrives;
+// outgrown areas are kept until exit because work that uses them may still be queued.
 struct ScratchArea {
     uint8_t* ptr = nullptr;
     size_t bytes = 0;
 };
 
-static enec_status get_scratch(int dev, cudaStream_t stream, size_t need, uint8_t** out) {
+enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1 };
+
+static enec_status get_scratch(int dev, cudaStream_t stream, ScratchKind kind, size_t need, uint8_t** out) {
     static std::mutex mu;
-    static std::map<std::pair<int, cudaStream_t>, ScratchArea> areas;
+    static std::map<std::pair<std::pair<int, int>, cudaStream_t>, ScratchArea> areas;
     std::lock_guard<std::mutex> lock(mu);
-    ScratchArea& a = areas[std::make_pair(dev, stream)];
+    ScratchArea& a = areas[std::make_pair(std::make_pair(dev, int(kind)), stream)];
     if (a.bytes < need) {
         size_t bytes = a.bytes ? a.bytes : size_t(64) << 10;
         while (bytes < need) bytes *= 2;
@@ -120,7 +122,7 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
     const Geometry g = make_geometry(count);
     const size_t need = kControlBytes + size_t(g.nblocks) * sizeof(unsigned long long);
     uint8_t* scratch = nullptr;
-    const enec_status st = get_scratch(dev, stream, need, &scratch);
+    const enec_status st = get_scratch(dev, stream, kScratchCompress, need, &scratch);
     if (st != ENEC_OK) return st;
     if (cudaMemsetAsync(scratch, 0, need, stream) != cudaSuccess) return ENEC_ERR_CUDA;
     EncodeJob job;
@@ -161,10 +163,59 @@ enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, siz
     if (!d_in || (!d_out && count) || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out))
         return ENEC_ERR_INVALID_ARG;
     if (in_size < kHeaderBytes + 16) return ENEC_ERR_BAD_STREAM;
-    DecodeJob job{static_cast<const uint8_t*>(d_in), static_cast<uint16_t*>(d_out), uint64_t(count), uint64_t(in_size)};
-    const Geometry g = make_geometry(count);
-    return dt == ENEC_BF16 ? launch_decode<ENEC_BF16>(job, g.nblocks, d_status, stream)
-                           : launch_decode<ENEC_FP16>(job, g.nblocks, d_status, stream);
+    DecodeBatch batch;
+    batch.jobs = nullptr;
+    batch.prefix = nullptr;
+    batch.n_jobs = 1;
+    batch.total_blocks = make_geometry(count).nblocks;
+    batch.single = DecodeJob{static_cast<const uint8_t*>(d_in), static_cast<uint16_t*>(d_out), uint64_t(count),
+                             uint64_t(in_size)};
+    return dt == ENEC_BF16 ? launch_decode<ENEC_BF16>(batch, d_status, stream)
+                           : launch_decode<ENEC_FP16>(batch, d_status, stream);
+}
+
+enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, int* d_status,
+                                    enec_stream_t stream) {
+    if (dt != ENEC_BF16 && dt != ENEC_FP16) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if (n_items < 0 || (n_items > 0 && !h_items)) return ENEC_ERR_INVALID_ARG;
+    if (n_items == 0) return ENEC_OK;
+    // descriptors and block prefix in one host buffer: [jobs | prefix]
+    const size_t jobs_bytes = size_t(n_items) * sizeof(DecodeJob);
+    const size_t prefix_bytes = (size_t(n_items) + 1) * sizeof(uint32_t);
+    std::vector<uint8_t> host(jobs_bytes + prefix_bytes);
+    DecodeJob* jobs = reinterpret_cast<DecodeJob*>(host.data());
+    uint32_t* prefix = reinterpret_cast<uint32_t*>(host.data() + jobs_bytes);
+    uint64_t total = 0;
+    for (int i = 0; i < n_items; ++i) {
+        const enec_batch_item& it = h_items[i];
+        if (!it.d_in || (!it.d_out && it.count) || (uint64_t(it.count) >> 36) || !aligned16(it.d_in) ||
+            !aligned16(it.d_out))
+            return ENEC_ERR_INVALID_ARG;
+        if (it.size < kHeaderBytes + 16) return ENEC_ERR_BAD_STREAM;
+        jobs[i] = DecodeJob{static_cast<const uint8_t*>(it.d_in), static_cast<uint16_t*>(it.d_out), uint64_t(it.count),
+                            uint64_t(it.size)};
+        prefix[i] = uint32_t(total);
+        total += make_geometry(it.count).nblocks;
+        if (total >> 31) return ENEC_ERR_INVALID_ARG;  // block indices are 32-bit
+    }
+    prefix[n_items] = uint32_t(total);
+    if (total == 0) return ENEC_OK;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
+    uint8_t* scratch = nullptr;
+    const enec_status st = get_scratch(dev, stream, kScratchBatch, host.size(), &scratch);
+    if (st != ENEC_OK) return st;
+    // pageable source: the call returns once the bytes are staged, so `host` may go out of scope
+    if (cudaMemcpyAsync(scratch, host.data(), host.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return ENEC_ERR_CUDA;
+    DecodeBatch batch;
+    batch.jobs = reinterpret_cast<const DecodeJob*>(scratch);
+    batch.prefix = reinterpret_cast<const uint32_t*>(scratch + jobs_bytes);
+    batch.n_jobs = uint32_t(n_items);
+    batch.total_blocks = uint32_t(total);
+    batch.single = DecodeJob{nullptr, nullptr, 0, 0};
+    return dt == ENEC_BF16 ? launch_decode<ENEC_BF16>(batch, d_status, stream)
+                           : launch_decode<ENEC_FP16>(batch, d_status, stream);
 }
 
 enec_status enec_compress(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
@@ -178,9 +229,6 @@ enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t co
     return compress_common(d_in, dt, count, true, b, n, m, d_out, out_capacity, d_out_size, d_status, stream);
 }
 
-enec_status enec_decompress_batched(const enec_batch_item*, int, enec_dtype, int*, enec_stream_t) {
-    return ENEC_ERR_CUDA;  // TEMP
-}
 
 uint64_t enec_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -17,9 +17,10 @@ namespace enec {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
-constexpr int kMaxStages = 4;
+constexpr int kStages = 2;
 constexpr uint32_t kDecodeSmemBytes = 75 * 1024;  // three CTAs per SM
-constexpr uint32_t kStageMetaBytes = 16;
+constexpr uint32_t kStageMetaBytes = 128;
+constexpr uint32_t kStageBytes = ((kDecodeSmemBytes - 128) / kStages) & ~15u;
 constexpr uint32_t kNotWide = 0xFFFFu;            // rank-array entry of a group stored with m bits
 
 // ---------------------------------------------------------------------------------------------------
@@ -207,37 +208,31 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
 }
 
 // Shared-memory layout of one pipeline stage (offsets from the stage base; all multiples of 16).
-//   meta | mask | rank array | low plane | fp16 sm-hi plane | sm bytes | raw records | expanded records
+//   descriptor | mask | rank array | low plane | fp16 sm-hi plane | sm bytes | raw records | expanded records
 // rank array: one u16 per group = rank of the group's record inside the block, or kNotWide.
 // expanded records: sixteen bytes per wide group (its high bits, one element per byte), rank order, and
-// one all-zero slot at index cap that the rank entries of narrow groups point to in blocks that fit.
+// one more slot at index cap that the rank entries of narrow groups point to in blocks that fit.
 // cap = records per block that fit; records beyond it are read from global memory by the consumers.
 struct StageLayout {
     uint32_t mask, rank, low, smhi, sm, raw, expanded, cap, bytes;
 };
-__device__ __forceinline__ StageLayout make_stage_layout(int dt, int m, int hbits, uint32_t budget, int& nstages) {
+__host__ __device__ inline StageLayout make_stage_layout(int dt, int m, int hbits) {
     StageLayout L;
     L.mask = kStageMetaBytes;
     L.rank = L.mask + kGroupsPerBlock / 8;
     L.low = L.rank + kGroupsPerBlock * 2;
     L.smhi = L.low + kBlockElems * uint32_t(m) / 8;
     L.sm = L.smhi + (dt == ENEC_FP16 ? kBlockElems * 3 / 8 : 0);
-    L.raw = L.sm + kBlockElems;
-    nstages = 2;
-    uint32_t per_stage = (budget / 2) & ~15u;
-    if (per_stage < L.raw + 64) { nstages = 1; per_stage = budget & ~15u; }
-    if (per_stage < L.raw + 64) { nstages = 0; per_stage = L.raw + 64; }
-    uint32_t cap = hbits > 0 ? (per_stage - L.raw - 64) / uint32_t(2 * hbits + 16) : 0;
+    L.raw = L.sm + kBlockElems;  // at most 35072 (m = 8, or fp16 with m = 5), so a stage always has room
+    uint32_t cap = hbits > 0 ? (kStageBytes - L.raw - 64) / uint32_t(2 * hbits + 16) : 0;
     if (cap > kGroupsPerBlock) cap = kGroupsPerBlock;
     L.cap = cap;
     L.expanded = L.raw + uint32_t(align16(uint64_t(cap) * 2 * hbits + 32));
     L.bytes = L.expanded + (cap + 1) * 16;
-    if (nstages == 2) {
-        int more = int(budget / L.bytes);
-        nstages = more > kMaxStages ? kMaxStages : more;
-    }
     return L;
 }
+static_assert(kStageMetaBytes + kGroupsPerBlock / 8 + kGroupsPerBlock * 2 + 2 * kBlockElems + 64 <= kStageBytes,
+              "the fixed part of the widest block fits a stage");
 
 struct RunCtx {
     uint32_t sm;          // shared address: sign/mantissa bytes of the block
@@ -500,8 +495,8 @@ __device__ __forceinline__ bool consumer_barrier_or(bool flag) {
 }
 
 struct DecodeShared {
-    uint64_t full[kMaxStages];   // bulk copies of a stage have landed
-    uint64_t empty[kMaxStages];  // all consumer warps are done with a stage
+    uint64_t full[4];   // bulk copies of a stage have landed (kStages used)
+    uint64_t empty[4];  // all consumer warps are done with a stage
     int abort;
     int pad[15];
 };
@@ -534,58 +529,117 @@ __device__ __forceinline__ bool poll_wait(uint64_t* bar, uint32_t parity, volati
     return false;
 }
 
+// What the loader tells the consumers about the block in a stage (first bytes of the stage).
+struct BlockDesc {
+    uint32_t first;     // offset of the block's first record inside the staged window
+    uint32_t staged;    // records staged in shared memory
+    uint32_t expect;    // wide groups of the block according to the prefix table
+    uint32_t N;         // padded block length
+    uint32_t real;      // real elements
+    uint32_t code;      // m * 8 + (n - m)
+    uint32_t b, n;
+    StageLayout L;
+    uint16_t* out;        // global: first element of the block
+    const uint8_t* high;  // global: first record of the block
+};
+static_assert(sizeof(BlockDesc) <= kStageMetaBytes, "descriptor fits the stage's meta area");
+
+// A launch decodes the blocks of one tensor or of a list of tensors. Blocks of all tensors form one
+// index space; a CTA takes a contiguous range of it, so it changes tensor rarely.
+struct DecodeBatch {
+    const DecodeJob* jobs;    // device array, or null for a single tensor
+    const uint32_t* prefix;   // device array [n_jobs + 1]: blocks before each tensor
+    uint32_t n_jobs;
+    uint32_t total_blocks;
+    DecodeJob single;         // the tensor when jobs is null
+};
+
 template <int DT>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
-enec_decode_kernel(DecodeJob job, int* status) {
+enec_decode_kernel(DecodeBatch batch, int* status) {
     extern __shared__ __align__(128) uint8_t smem[];
     DecodeShared* ctl = reinterpret_cast<DecodeShared*>(smem);
     const uint32_t stages = smem_u32(smem) + uint32_t(sizeof(DecodeShared));
+    constexpr uint32_t S = kStages;
 
-    JobCtx jc;
-    const int err = load_job<DT>(job, jc);
-    if (err) {
-        if (threadIdx.x == 0 && blockIdx.x == 0) report(status, err);
-        return;
-    }
-    const int hbits = jc.n - jc.m;
-    int nstages = 0;
-    const StageLayout L = make_stage_layout(DT, jc.m, hbits, kDecodeSmemBytes - uint32_t(sizeof(DecodeShared)), nstages);
-    if (nstages < 1) {  // cannot happen for valid (m, n): the fixed part of a stage is below 40 KB
-        if (threadIdx.x == 0 && blockIdx.x == 0) report(status, ENEC_ERR_BAD_STREAM);
+    if (batch.total_blocks == 0) {  // nothing to decode: only check the header of a single empty tensor
+        if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr) {
+            JobCtx jc;
+            const int err = load_job<DT>(batch.single, jc);
+            if (err) report(status, err);
+        }
         return;
     }
     if (threadIdx.x == 0) {
-        for (int s = 0; s < nstages; ++s) {
+        for (uint32_t s = 0; s < S; ++s) {
             mbar_init(&ctl->full[s], 1);
             mbar_init(&ctl->empty[s], kConsumerWarps);
         }
         ctl->abort = 0;
         mbar_fence_init();
     }
-    // the slot narrow groups point to in the branch-free body: no high bits, sign position flipped
-    const uint32_t flip4 = hbits > 0 ? rep4(1u << (hbits - 1)) : 0;
-    if (threadIdx.x < uint32_t(nstages))
-        sts128(stages + threadIdx.x * L.bytes + L.expanded + L.cap * 16, make_uint4(flip4, flip4, flip4, flip4));
     __syncthreads();
 
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lane = threadIdx.x & 31;
     volatile int* abort_flag = &ctl->abort;
-    const uint32_t n_mine = jc.nblocks > blockIdx.x ? (jc.nblocks - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-    const uint32_t S = uint32_t(nstages);
-    const uint32_t* table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
+    const uint32_t first_block = uint32_t(uint64_t(blockIdx.x) * batch.total_blocks / gridDim.x);
+    const uint32_t end_block = uint32_t(uint64_t(blockIdx.x + 1) * batch.total_blocks / gridDim.x);
+    const uint32_t n_mine = end_block - first_block;
 
     if (warp == kConsumerWarps) {
         // ---------------- loader warp: lane 0 issues the copies of block after block ----------------
         if (lane != 0) return;
+        // the tensor that holds first_block
+        uint32_t j = 0;
+        if (batch.jobs) {
+            uint32_t lo = 0, hi = batch.n_jobs;  // largest j with prefix[j] <= first_block
+            while (hi - lo > 1) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (batch.prefix[mid] <= first_block) lo = mid; else hi = mid;
+            }
+            j = lo;
+        }
+        uint32_t job_first = batch.jobs ? batch.prefix[j] : 0;
+        uint32_t job_end = batch.jobs ? batch.prefix[j + 1] : batch.total_blocks;
+        bool parsed = false;
+        JobCtx jc;
+        StageLayout L;
+        int hbits = 0;
+        const uint32_t* table = nullptr;
+        uint32_t t1 = 0, t2 = 0;  // table[k + 1], table[k + 2] of the block about to be issued (one ahead)
         uint32_t issued = 0;
         bool failed = false;
-        uint32_t t0 = 0, t1 = 0;  // table entries of the next block to issue, fetched one block ahead
-        if (n_mine) { t0 = table[blockIdx.x]; t1 = table[blockIdx.x + 1]; }
         for (; issued < n_mine; ++issued) {
+            const uint32_t gb = first_block + issued;
+            while (gb >= job_end) {  // next tensor (tensors without blocks are skipped)
+                ++j;
+                job_first = job_end;
+                job_end = batch.prefix[j + 1];
+                parsed = false;
+            }
+            const uint32_t k = gb - job_first;
+            uint32_t t0;
+            if (!parsed) {
+                const int err = load_job<DT>(batch.jobs ? batch.jobs[j] : batch.single, jc);
+                if (err) {
+                    *abort_flag = 1;
+                    report(status, err);
+                    failed = true;
+                    break;
+                }
+                hbits = jc.n - jc.m;
+                L = make_stage_layout(DT, jc.m, hbits);
+                table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
+                t0 = table[k];
+                t1 = table[k + 1];
+                parsed = true;
+            } else {
+                t0 = t1;
+                t1 = t2;
+            }
             const uint32_t s = issued % S, use = issued / S;
             if (use > 0 && !poll_wait(&ctl->empty[s], (use - 1) & 1, abort_flag)) { failed = true; break; }
-            const uint32_t k = blockIdx.x + issued * gridDim.x;
             const bool tail = (k + 1 == jc.nblocks);
             const uint32_t N = tail ? jc.tail_padded : kBlockElems;
             const uint32_t real = tail ? jc.tail_real : kBlockElems;
@@ -605,12 +659,19 @@ enec_decode_kernel(DecodeJob job, int* status) {
             const uint32_t smhi_bytes = DT == ENEC_FP16 ? uint32_t(align16(uint64_t(N) * 3 / 8)) : 0;
             const uint32_t sm_bytes = uint32_t(align16(real));
             const uint32_t raw_bytes = staged ? uint32_t(w1 - w0) : 0;
-            uint8_t* st = smem + sizeof(DecodeShared) + size_t(s) * L.bytes;
-            uint32_t* meta = reinterpret_cast<uint32_t*>(st);
-            meta[0] = uint32_t(h0 - w0);  // offset of the first record inside the staged window
-            meta[1] = staged;
-            meta[2] = t1 - t0;
-            meta[3] = t0;
+            uint8_t* st = smem + sizeof(DecodeShared) + size_t(s) * kStageBytes;
+            BlockDesc* d = reinterpret_cast<BlockDesc*>(st);
+            d->first = uint32_t(h0 - w0);
+            d->staged = staged;
+            d->expect = t1 - t0;
+            d->N = N;
+            d->real = real;
+            d->code = uint32_t(jc.m * 8 + hbits);
+            d->b = uint32_t(jc.b);
+            d->n = uint32_t(jc.n);
+            d->L = L;
+            d->out = jc.out + uint64_t(k) * kBlockElems;
+            d->high = jc.in + h0;
             mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes);
             bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
             bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
@@ -618,7 +679,7 @@ enec_decode_kernel(DecodeJob job, int* status) {
                 bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
             bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
             if (raw_bytes) bulk_g2s(st + L.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
-            if (issued + 1 < n_mine) { t0 = table[k + gridDim.x]; t1 = table[k + gridDim.x + 1]; }
+            if (k + 2 <= jc.nblocks) t2 = table[k + 2];  // for the tensor's next block
         }
         if (failed) {
             if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
@@ -630,26 +691,10 @@ enec_decode_kernel(DecodeJob job, int* status) {
     }
 
     // ---------------- consumers ----------------
-    RunCtx r;
-    {
-        const uint32_t sbit = 1u << (jc.n - 1);
-        const uint32_t c = (uint32_t(jc.b) + sbit) & 0xFF;
-        r.s4 = rep4(sbit);
-        r.c4_or_h = rep4(c) | 0x80808080u;
-        r.fix = ~rep4(c) & 0x80808080u;
-        r.b4 = rep4(uint32_t(jc.b));
-        r.c4 = rep4(c);
-        r.n = jc.n;
-        r.cap = L.cap;
-    }
-    const int code = jc.m * 8 + hbits;
     const uint32_t tid = threadIdx.x;
     for (uint32_t i = 0; i < n_mine; ++i) {
         const uint32_t s = i % S, use = i / S;
-        const uint32_t k = blockIdx.x + i * gridDim.x;
-        const bool tail = (k + 1 == jc.nblocks);
-        const uint32_t N = tail ? jc.tail_padded : kBlockElems;
-        const uint32_t st = stages + s * L.bytes;
+        const uint32_t st = stages + s * kStageBytes;
         // one thread waits for the block's bytes; the others sleep at the barrier
         bool failed = false;
         if (tid == 0 && !poll_wait(&ctl->full[s], use & 1, abort_flag)) {
@@ -659,39 +704,59 @@ enec_decode_kernel(DecodeJob job, int* status) {
         // every consumer reaches both barriers of a block, failed wait or not, and all leave together
         if (consumer_barrier_or(failed || *abort_flag != 0)) break;
         mbar_try_wait(&ctl->full[s], use & 1);  // completed: acquires the copied bytes in every thread
+        const BlockDesc* d = reinterpret_cast<const BlockDesc*>(smem + sizeof(DecodeShared) + size_t(s) * kStageBytes);
+        const uint32_t N = d->N, expect = d->expect, code = d->code;
+        const uint32_t b = d->b, n = d->n;
+        const uint32_t hbits = code & 7;
+        const uint32_t cap = d->L.cap;
+        const uint32_t o_rank = d->L.rank, o_low = d->L.low, o_smhi = d->L.smhi, o_sm = d->L.sm, o_raw = d->L.raw,
+                       o_exp = d->L.expanded;
+        const uint32_t sbit = 1u << (n - 1);
+        const bool simple_sub = DT == ENEC_FP16 || n == 8 || b + sbit <= 255;
+        const bool full_block = N == kBlockElems && d->real == kBlockElems && expect <= cap && simple_sub;
         // preparation: ranks of the wide groups and expanded records
-        const uint32_t first = lds32(st), staged = lds32(st + 4), expect = lds32(st + 8);
-        const bool simple_sub = DT == ENEC_FP16 || jc.n == 8 || uint32_t(jc.b) + (1u << (jc.n - 1)) <= 255;
-        const bool full_block = !tail && expect <= L.cap && simple_sub;
         if (hbits > 0) {
             // the branch-free body wants narrow groups to point at the flip slot and flipped records
-            const uint32_t wide = build_rank_array(st + L.mask, st + L.rank, N, tid, full_block ? L.cap : kNotWide);
+            const uint32_t flip4 = rep4(1u << (hbits - 1));
+            if (tid == 0) sts128(st + o_exp + cap * 16, make_uint4(flip4, flip4, flip4, flip4));
+            const uint32_t wide = build_rank_array(st + d->L.mask, st + o_rank, N, tid, full_block ? cap : kNotWide);
             if (wide != expect && lane == 0) {  // the prefix table must agree with the mask
                 *abort_flag = 1;
                 report(status, ENEC_ERR_BAD_STREAM);
             }
-            expand_records_any(hbits, st + L.raw + first, st + L.expanded, staged, tid, full_block ? flip4 : 0);
+            expand_records_any(int(hbits), st + o_raw + d->first, st + o_exp, d->staged, tid, full_block ? flip4 : 0);
         }
-        r.high = jc.in + jc.off_high + uint64_t(lds32(st + 12)) * (2 * hbits);
+        RunCtx r;
+        {
+            const uint32_t c = (b + sbit) & 0xFF;
+            r.s4 = rep4(sbit);
+            r.c4_or_h = rep4(c) | 0x80808080u;
+            r.fix = ~rep4(c) & 0x80808080u;
+            r.b4 = rep4(b);
+            r.c4 = rep4(c);
+            r.n = int(n);
+            r.cap = cap;
+            r.sm = st + o_sm;
+            r.rank = st + o_rank;
+            r.expanded = st + o_exp;
+            r.out = d->out;
+            r.high = d->high;
+            r.real = d->real;
+        }
         if (consumer_barrier_or(*abort_flag != 0)) break;
-        r.sm = st + L.sm;
-        r.rank = st + L.rank;
-        r.expanded = st + L.expanded;
-        r.out = jc.out + uint64_t(k) * kBlockElems;
-        r.real = tail ? jc.tail_real : kBlockElems;
         switch (code) {
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
-        if (full_block) decode_full_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, tid);     \
-        else decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, tid);                  \
+        if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid);     \
+        else decode_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, N, tid);                  \
         break;
             ENEC_FOR_EACH_MH(ENEC_CASE, DT)
 #undef ENEC_CASE
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
         if constexpr (DTV == ENEC_BF16) {                                                    \
-            if (full_block) decode_full_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, tid); \
-            else decode_block<DTV, MV, HV>(r, st + L.low, st + L.smhi, N, tid);              \
+            if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid); \
+            else decode_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, N, tid);              \
         }                                                                                    \
         break;
             ENEC_FOR_EACH_MH_BF16_ONLY(ENEC_CASE, DT)

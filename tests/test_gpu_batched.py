@@ -1,0 +1,101 @@
+"""GPU parity of enec_decompress_batched: many streams, one launch, every tensor bit-exact (tolerance 0)."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import status_tensor, tensor_of, to_dev_bytes, words_of
+
+pytestmark = pytest.mark.gpu
+
+DT = {0: torch.bfloat16, 1: torch.float16}
+
+
+def _words(rng, count, dt, spread):
+    E, mant = (8, 7) if dt == 0 else (5, 10)
+    center = 120 if dt == 0 else 12
+    x = np.clip(np.round(rng.normal(center, spread, count)), 0, (1 << E) - 1).astype(np.uint16)
+    return ((x << mant) | rng.integers(0, 1 << mant, count).astype(np.uint16)
+            | (rng.integers(0, 2, count).astype(np.uint16) << 15)).astype(np.uint16)
+
+
+@pytest.mark.parametrize("dt", [0, 1])
+def test_mixed_batch_against_oracle_streams(oracle, dt):
+    import paper_2604_03298_b200 as enec
+    rng = np.random.default_rng(40 + dt)
+    counts = [16384 * 7 + 5, 0, 1, 16, 2048, 16384, 100, 16384 * 30, 17, 16384 * 3 + 8000, 0, 40, 16384 * 2 + 1] + [2048] * 40
+    spreads = [0.4, 1.0, 2.0, 4.0, 30.0]
+    items, wants = [], []
+    for i, c in enumerate(counts):
+        w = _words(rng, c, dt, spreads[i % len(spreads)])       # different (b, n, m) per tensor
+        s = oracle.compress(w, dt)
+        d_in = to_dev_bytes(s)
+        guard = torch.full((c + 64,), 0x5A5A, dtype=torch.int16, device="cuda")
+        items.append((d_in, d_in.numel(), guard, c))
+        wants.append(w)
+    status = status_tensor()
+    call = [(src, nbytes, g[:c].view(DT[dt]) if c else g[:0].view(DT[dt]), c) for src, nbytes, g, c in items]
+    before = enec.enec_launch_count()
+    assert enec.enec_decompress_batched(call, dt, status) == 0
+    torch.cuda.synchronize()
+    assert enec.enec_launch_count() - before == 1
+    assert int(status.item()) == 0
+    for (src, nbytes, g, c), w in zip(items, wants):
+        assert (g[c:] == 0x5A5A).all()
+        got = g[:c].cpu().numpy().view(np.uint16)
+        assert np.array_equal(got, w)
+
+
+def test_moe_shaped_set_full_size():
+    """Workload 5 at full size (768 expert matrices + 4096 vectors of 2048, bf16): streams written by enec_compress
+    (checked byte for byte against the oracle elsewhere), all decompressed by one batched launch."""
+    import paper_2604_03298_b200 as enec
+    from paper_2604_03298_b200 import runner, synth
+    specs = synth.config_specs(5)
+    assert len(specs) == 768 + 4096
+    # the expert matrices share three shapes and one distribution: draw 24 distinct ones and reuse them
+    distinct = {}
+    raw = []
+    for i, s in enumerate(specs):
+        key = (s.shape, i % 24) if len(s.shape) == 2 else ("v", i)
+        if key not in distinct:
+            distinct[key] = synth.make_tensor(s, "cuda")
+        raw.append(distinct[key])
+    cs = runner.CodecSet.allocate(raw)
+    cs.compress_all()
+    torch.cuda.synchronize()
+    cs.check_status()
+    sizes = cs.sizes.cpu().tolist()
+    items = [(cs.streams[i], sizes[i], cs.outs[i], raw[i].numel()) for i in range(len(raw))]
+    before = enec.enec_launch_count()
+    assert enec.enec_decompress_batched(items, 0, cs.status) == 0
+    torch.cuda.synchronize()
+    assert enec.enec_launch_count() - before == 1
+    cs.check_status()
+    cs.verify_roundtrip()
+
+
+def test_damaged_member_is_reported(oracle):
+    import paper_2604_03298_b200 as enec
+    rng = np.random.default_rng(50)
+    streams = [oracle.compress(_words(rng, 16384 * 4 + 9, 0, 2.0), 0) for _ in range(6)]
+    streams[3] = streams[3].copy()
+    streams[3][22] = 9                                   # m beyond n
+    call = []
+    for s in streams:
+        d = to_dev_bytes(s)
+        call.append((d, d.numel(), torch.empty(16384 * 4 + 9, dtype=torch.bfloat16, device="cuda"), 16384 * 4 + 9))
+    status = status_tensor()
+    assert enec.enec_decompress_batched(call, 0, status) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == -4
+
+
+def test_host_argument_checks():
+    import paper_2604_03298_b200 as enec
+    buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(64, dtype=torch.bfloat16, device="cuda")
+    assert enec.enec_decompress_batched([], 0) == 0
+    assert enec.enec_decompress_batched([(buf, 4096, out, 64)], 9) == -2
+    assert enec.enec_decompress_batched([(buf[1:], 4000, out, 64)], 0) == -1
+    assert enec.enec_decompress_batched([(buf, 10, out, 64)], 0) == -4
+    torch.cuda.synchronize()
