@@ -40,7 +40,8 @@ typedef enum {
     ENEC_ERR_BAD_STREAM = -4,
     ENEC_ERR_PARAMS_NOT_LOSSLESS = -5,
     ENEC_ERR_TIMEOUT = -6,
-    ENEC_ERR_CUDA = -7
+    ENEC_ERR_CUDA = -7,
+    ENEC_ERR_TOO_LARGE = -8
 } enec_status;
 
 /* Same type as cudaStream_t; spelled out so that this header needs no CUDA header. */
@@ -100,6 +101,35 @@ typedef struct {
  */
 enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, int* d_status,
                                     enec_stream_t stream);
+
+/*
+ * enec_compress for callers that must not allocate device memory. (The paper has no counterpart: this is
+ * a property of this library's interface, not of the codec.)
+ *
+ * enec_compress keeps its working memory (a histogram, a few control words and one 8-byte word per
+ * 16384-value block) in an area it allocates with cudaMalloc the first time a stream is used, and again
+ * when a larger tensor arrives. Some callers cannot have that: code that runs inside a memory pool or a
+ * caching allocator which owns all device memory and must see every allocation, code in a phase where a
+ * cudaMalloc would stall other streams (it synchronises the device), and services that have handed the
+ * whole device budget to something else. For them this entry point takes its working memory from a
+ * fixed array inside the library image (ENEC_NOALLOC_SCRATCH_BYTES, about 0.5 MB, present on every GPU
+ * that loads the library for as long as the process lives) and calls neither cudaMalloc nor cudaFree
+ * nor any routine that allocates.
+ *
+ * Same arguments, stream format and output as enec_compress (the two write identical bytes). Limits and
+ * rules that differ:
+ *   - count may be at most ENEC_NOALLOC_MAX_COUNT (2^30 values, 2 GiB of bf16); more is refused with
+ *     ENEC_ERR_TOO_LARGE before anything is enqueued. Split larger tensors or use enec_compress.
+ *   - All calls on a device share the one array, whatever their stream. Each call begins by clearing the
+ *     part it uses, so calls that follow one another on a stream are fine; two calls whose work overlaps
+ *     on the GPU (different streams without an ordering between them) corrupt each other's state.
+ *   - The first call on each device looks up the array's device address, with that device current. Make
+ *     that first call outside any stream capture.
+ */
+#define ENEC_NOALLOC_MAX_COUNT ((size_t)1 << 30)
+#define ENEC_NOALLOC_SCRATCH_BYTES (4096 + (ENEC_NOALLOC_MAX_COUNT / 16384) * 8)
+enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                                  size_t* d_out_size, int* d_status, enec_stream_t stream);
 
 /* Number of kernels the library has launched in this process (all entry points, all streams). */
 uint64_t enec_launch_count(void);

@@ -13,7 +13,8 @@ _DT = {torch.bfloat16: BF16, torch.float16: FP16}
 
 STATUS_NAMES = {0: "ENEC_OK", -1: "ENEC_ERR_INVALID_ARG", -2: "ENEC_ERR_UNSUPPORTED_DTYPE",
                 -3: "ENEC_ERR_BUFFER_TOO_SMALL", -4: "ENEC_ERR_BAD_STREAM",
-                -5: "ENEC_ERR_PARAMS_NOT_LOSSLESS", -6: "ENEC_ERR_TIMEOUT", -7: "ENEC_ERR_CUDA"}
+                -5: "ENEC_ERR_PARAMS_NOT_LOSSLESS", -6: "ENEC_ERR_TIMEOUT", -7: "ENEC_ERR_CUDA",
+                -8: "ENEC_ERR_TOO_LARGE"}
 
 
 class EnecError(RuntimeError):
@@ -39,6 +40,8 @@ def lib():
         L.enec_compress.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p,
                                     C.c_void_p, C.c_void_p]
         L.enec_compress.restype = C.c_int
+        L.enec_compress_noalloc.argtypes = L.enec_compress.argtypes
+        L.enec_compress_noalloc.restype = C.c_int
         L.enec_compress_with_params.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_int,
                                                 C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
         L.enec_compress_with_params.restype = C.c_int
@@ -71,6 +74,13 @@ def enec_compress(d_in, dt, count, d_out, out_capacity, d_out_size=None, d_statu
     """d_in/d_out/d_out_size/d_status: CUDA tensors (or None). Enqueues on the current stream; returns status."""
     return lib().enec_compress(_ptr(d_in), dt, count, _ptr(d_out), out_capacity, _ptr(d_out_size),
                                _ptr(d_status), _stream())
+
+
+def enec_compress_noalloc(d_in, dt, count, d_out, out_capacity, d_out_size=None, d_status=None) -> int:
+    """enec_compress with the library's built-in scratch array instead of allocated scratch: for callers that
+    must not allocate device memory. At most 2^30 values; calls that overlap on the GPU must not share a device."""
+    return lib().enec_compress_noalloc(_ptr(d_in), dt, count, _ptr(d_out), out_capacity, _ptr(d_out_size),
+                                       _ptr(d_status), _stream())
 
 
 def enec_compress_with_params(d_in, dt, count, b, n, m, d_out, out_capacity, d_out_size=None, d_status=None) -> int:

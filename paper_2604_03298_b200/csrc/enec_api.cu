@@ -139,6 +139,30 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
                            : launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream);
 }
 
+// ---- compression without any allocation ------------------------------------------------------------
+// Scratch of enec_compress_noalloc: the compressor's control words and one look-back state word per
+// block, for tensors of up to kNoAllocMaxCount values, held in the library image on every GPU that loads
+// it. In host code `g_noalloc_scratch` is only a handle for cudaGetSymbolAddress, never an address to
+// hand to a kernel.
+constexpr uint64_t kNoAllocMaxCount = uint64_t(1) << 30;
+constexpr size_t kNoAllocScratchBytes = kControlBytes + size_t(kNoAllocMaxCount / kBlockElems) * sizeof(unsigned long long);
+static __device__ __align__(256) uint8_t g_noalloc_scratch[kNoAllocScratchBytes];
+
+// Device address of the scratch on the current device, looked up once per device.
+static enec_status noalloc_scratch(int dev, uint8_t** out) {
+    static std::mutex mu;
+    static uint8_t* addr[64] = {};
+    if (dev < 0 || dev >= 64) return ENEC_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return ENEC_ERR_CUDA;
+        addr[dev] = static_cast<uint8_t*>(p);
+    }
+    *out = addr[dev];
+    return ENEC_OK;
+}
+
 }  // namespace enec
 
 using namespace enec;
@@ -229,6 +253,44 @@ enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t co
     return compress_common(d_in, dt, count, true, b, n, m, d_out, out_capacity, d_out_size, d_status, stream);
 }
 
+
+enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                                  size_t* d_out_size, int* d_status, enec_stream_t stream) {
+    if (dt != ENEC_BF16 && dt != ENEC_FP16) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if (uint64_t(count) > kNoAllocMaxCount) return ENEC_ERR_TOO_LARGE;
+    if ((!d_in && count) || !d_out || !aligned16(d_in) || !aligned16(d_out) ||
+        (reinterpret_cast<uintptr_t>(d_out_size) & 7))
+        return ENEC_ERR_INVALID_ARG;
+    if (out_capacity < enec_max_compressed_size(dt, count)) return ENEC_ERR_BUFFER_TOO_SMALL;
+    unsigned long long* out_size = reinterpret_cast<unsigned long long*>(d_out_size);
+    if (count == 0) {
+        enec_encode_empty_kernel<<<1, 32, 0, stream>>>(static_cast<uint8_t*>(d_out), int(dt), 0, 1, 1, out_size);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
+    uint8_t* scratch = nullptr;
+    const enec_status st = noalloc_scratch(dev, &scratch);
+    if (st != ENEC_OK) return st;
+    DeviceInfo& info = device_info(dev);
+    const Geometry g = make_geometry(count);
+    // the area keeps the previous call's words: histogram, ticket, flags and state words start at zero
+    const size_t used = kControlBytes + size_t(g.nblocks) * sizeof(unsigned long long);
+    if (cudaMemsetAsync(scratch, 0, used, stream) != cudaSuccess) return ENEC_ERR_CUDA;
+    EncodeJob job;
+    job.in = static_cast<const uint16_t*>(d_in);
+    job.out = static_cast<uint8_t*>(d_out);
+    job.count = count;
+    job.ctl = reinterpret_cast<EncodeControl*>(scratch);
+    job.state = reinterpret_cast<unsigned long long*>(scratch + kControlBytes);
+    job.out_size = out_size;
+    job.b = 0; job.n = 0; job.m = 0;
+    job.from_search = 1;
+    job.check = 0;
+    return dt == ENEC_BF16 ? launch_encode<ENEC_BF16>(job, g.nblocks, true, d_status, info, stream)
+                           : launch_encode<ENEC_FP16>(job, g.nblocks, true, d_status, info, stream);
+}
 
 uint64_t enec_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
