@@ -66,7 +66,7 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p) {
 //
 // Each lane keeps private 8-bit counters in shared memory (four bins per 32-bit word, the word's bank
 // equal to the lane), so counting needs neither atomics nor bank conflicts whatever the distribution;
-// a warp folds its counters into the CTA's 32-bit histogram every 31 loads of eight values (248 < 256).
+// a warp folds its counters into the CTA's 32-bit histogram every 28 loads of eight values (224 < 256).
 // ---------------------------------------------------------------------------------------------------
 template <int DT>
 struct HistShape {
@@ -222,18 +222,29 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
 
     const uint64_t nchunks = count >> 3;  // 16-byte loads of eight values
     const uint4* in4 = reinterpret_cast<const uint4*>(in);
-    const uint64_t stride = uint64_t(gridDim.x) * kHistThreads;
+    // a warp takes 2 KB at a time: four 16-byte loads per lane in flight before any counting
+    constexpr uint32_t kUnroll = 4;
+    const uint64_t warps_total = uint64_t(gridDim.x) * (kHistThreads / 32);
     uint32_t since_flush = 0;
-    for (uint64_t first = uint64_t(blockIdx.x) * kHistThreads + (tid & ~31u); first < nchunks; first += stride) {
-        const uint64_t i = first + lane;
-        if (i < nchunks) {
-            const uint4 v = in4[i];  // default caching: the encode pass reads the tensor again
-            count_word_pair<DT>(base, v.x);
-            count_word_pair<DT>(base, v.y);
-            count_word_pair<DT>(base, v.z);
-            count_word_pair<DT>(base, v.w);
+    for (uint64_t first = (uint64_t(blockIdx.x) * (kHistThreads / 32) + warp) * (32 * kUnroll); first < nchunks;
+         first += warps_total * (32 * kUnroll)) {
+        uint4 v[kUnroll];
+#pragma unroll
+        for (uint32_t u = 0; u < kUnroll; ++u) {
+            const uint64_t i = first + u * 32 + lane;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (i < nchunks) v[u] = in4[i];  // default caching: the encode pass reads the tensor again
         }
-        if (++since_flush == 31) {
+#pragma unroll
+        for (uint32_t u = 0; u < kUnroll; ++u) {
+            if (first + u * 32 + lane < nchunks) {
+                count_word_pair<DT>(base, v[u].x);
+                count_word_pair<DT>(base, v[u].y);
+                count_word_pair<DT>(base, v[u].z);
+                count_word_pair<DT>(base, v[u].w);
+            }
+        }
+        if (++since_flush == 7) {  // 7 * 4 * 8 = 224 values per lane since the last flush, below 256
             flush_counters<DT>(warp_base, lane, cta_hist);
             since_flush = 0;
         }
@@ -473,6 +484,65 @@ struct EncodeShared {
     uint32_t poisoned;
 };
 
+// Phase 1 of a full block (16384 real elements), all 256 threads: loads, split, transform, sign/mantissa
+// stores and group widths with immediate offsets and no bounds logic. Lanes l and l + 16 share a group, so
+// the two halves of a ballot OR into the mask of the warp's sixteen groups of run c.
+// SIMPLE (n < 8 and no loss check): only the low seven bits of b - x matter, so the exponent is taken
+// without its top bit and a guard bit absorbs the borrow: y = ((b & 127 | 128) - (x & 127)) & (2^n - 1).
+// Returns the wide flags of the thread's eight runs (bit c).
+template <int DT, bool SIMPLE>
+__device__ __forceinline__ uint32_t encode_full_runs(const uint16_t* in_thread, uint8_t* sm_thread, const TransformCtx& tc,
+                                                     int m, uint32_t warp, uint32_t lane, uint32_t* mask_words,
+                                                     uint2 (&y)[8], uint2 (&hs)[8], int& bad) {
+    constexpr uint32_t kRunStride = kBlockElems / 8;  // elements between a thread's runs
+    uint4 raw[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) raw[c] = __ldcs(reinterpret_cast<const uint4*>(in_thread + c * kRunStride));
+    const uint32_t c7 = (tc.b4 & 0x7F7F7F7Fu) | 0x80808080u;
+    const uint32_t widemask4 = ~rep4((1u << m) - 1);
+    uint32_t wide_bits = 0;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint32_t sm0, sm1;
+        if constexpr (SIMPLE) {
+            const uint32_t lo0 = prmt(raw[c].x, raw[c].y, 0x6420u), hi0 = prmt(raw[c].x, raw[c].y, 0x7531u);
+            const uint32_t lo1 = prmt(raw[c].z, raw[c].w, 0x6420u), hi1 = prmt(raw[c].z, raw[c].w, 0x7531u);
+            uint32_t x0, x1;  // exponent fields without bit 7
+            if (DT == ENEC_BF16) {
+                x0 = ((hi0 << 1) & 0x7E7E7E7Eu) | ((lo0 >> 7) & 0x01010101u);
+                x1 = ((hi1 << 1) & 0x7E7E7E7Eu) | ((lo1 >> 7) & 0x01010101u);
+                sm0 = (hi0 & 0x80808080u) | (lo0 & 0x7F7F7F7Fu);
+                sm1 = (hi1 & 0x80808080u) | (lo1 & 0x7F7F7F7Fu);
+                hs[c] = make_uint2(0, 0);
+            } else {
+                x0 = (hi0 >> 2) & 0x1F1F1F1Fu;
+                x1 = (hi1 >> 2) & 0x1F1F1F1Fu;
+                sm0 = lo0;
+                sm1 = lo1;
+                hs[c] = make_uint2(((hi0 >> 5) & 0x04040404u) | (hi0 & 0x03030303u),
+                                   ((hi1 >> 5) & 0x04040404u) | (hi1 & 0x03030303u));
+            }
+            y[c] = make_uint2((c7 - x0) & tc.nmask4, (c7 - x1) & tc.nmask4);
+        } else {
+            const Split4 s0 = split4<DT>(raw[c].x, raw[c].y);
+            const Split4 s1 = split4<DT>(raw[c].z, raw[c].w);
+            const uint32_t d0 = bytewise_b_minus(tc, s0.x), d1 = bytewise_b_minus(tc, s1.x);
+            y[c] = make_uint2(d0 & tc.nmask4, d1 & tc.nmask4);
+            hs[c] = make_uint2(s0.hs, s1.hs);
+            bad |= (lossy_bytes(tc, d0, y[c].x) | lossy_bytes(tc, d1, y[c].y)) != 0;
+            sm0 = s0.sm;
+            sm1 = s1.sm;
+        }
+        __stcs(reinterpret_cast<uint2*>(sm_thread + c * kRunStride), make_uint2(sm0, sm1));
+        const bool wide_half = ((y[c].x | y[c].y) & widemask4) != 0;  // some value of this half needs more than m bits
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, wide_half);
+        const uint32_t groups16 = (bal | (bal >> 16)) & 0xFFFFu;
+        wide_bits |= ((groups16 >> (lane & 15)) & 1u) << c;
+        if (lane == 0) reinterpret_cast<uint16_t*>(mask_words)[c * 8 + warp] = uint16_t(groups16);
+    }
+    return wide_bits;
+}
+
 // Blocks shorter than 128 elements (16, 32 or 64): one element per thread, bits placed one by one.
 template <int DT>
 __device__ __noinline__ int encode_short_block(const uint16_t* in, uint32_t N, uint32_t real, const TransformCtx& tc,
@@ -550,7 +620,7 @@ enec_encode_kernel(EncodeJob job, int* status) {
     constexpr int E = DT == ENEC_BF16 ? 8 : 5;
     __shared__ __align__(16) uint8_t s_low[kBlockElems];                              // normalised bytes, low plane
     __shared__ __align__(16) uint8_t s_hi3[DT == ENEC_FP16 ? kBlockElems * 3 / 8 : 32];  // fp16 sign/mantissa-high plane
-    __shared__ __align__(16) uint8_t s_rec[kGroupsPerBlock * 14];                     // records of the block, rank order
+    __shared__ __align__(16) uint8_t s_rec[kGroupsPerBlock * 16];  // wide groups in rank order: 16 value bytes, then packed
     __shared__ EncodeShared sh;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -588,7 +658,7 @@ enec_encode_kernel(EncodeJob job, int* status) {
     int bad = 0;
     uint2 y[8];
     uint32_t wide_bits = 0;  // bit c: the group of run c is wide
-    const bool fast = N == kBlockElems;
+    const bool fast = N == kBlockElems && real == kBlockElems;
     // fast path: lanes l and l + 16 share a group, so a ballot's low half is the mask of sixteen groups
     const uint32_t perm = fast ? (warp * 32 + 2 * (lane & 15) + (lane >> 4)) : tid;
     const uint32_t pair_delta = fast ? 16 : 1;
@@ -597,11 +667,21 @@ enec_encode_kernel(EncodeJob job, int* status) {
     const uint32_t j = 8 * perm;
     const bool active = N >= 128 && perm < (N >> 6);
 
-    if (N >= 128) {
-        if (!fast) {
-            if (tid < 32) sh.mask[tid] = 0;
-            __syncthreads();
-        }
+    uint2 hs[8];
+    if (fast) {
+        if (!job.check && n < 8)
+            wide_bits = encode_full_runs<DT, true>(in + j, out_sm + j, tc, m, warp, lane, sh.mask, y, hs, bad);
+        else
+            wide_bits = encode_full_runs<DT, false>(in + j, out_sm + j, tc, m, warp, lane, sh.mask, y, hs, bad);
+        uint2 ylow[8];
+        const uint32_t lowmask4 = rep4((1u << m) - 1);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) ylow[c] = make_uint2(y[c].x & lowmask4, y[c].y & lowmask4);
+        pack_plane_any(m, smem_u32(s_low), j, N, ylow);
+        if (DT == ENEC_FP16) pack_plane<3>(smem_u32(s_hi3), j, N, hs);
+    } else if (N >= 128) {
+        if (tid < 32) sh.mask[tid] = 0;
+        __syncthreads();
         uint4 raw[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -617,7 +697,6 @@ enec_encode_kernel(EncodeJob job, int* status) {
                 }
             }
         }
-        uint2 hs[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             const uint32_t e0 = c * n8 + j;
@@ -703,20 +782,32 @@ enec_encode_kernel(EncodeJob job, int* status) {
         const uint32_t mask_vecs = uint32_t(align16(((N >> 4) + 7) / 8)) / 16;
         if (tid < mask_vecs)
             reinterpret_cast<uint4*>(out_mask)[tid] = reinterpret_cast<const uint4*>(sh.mask)[tid];
-        // records of wide groups into shared memory, rank order
+        // high bits of wide groups into shared memory, rank order, sixteen value bytes per group:
+        // each lane of a pair stores its own half
         if (hbits > 0) {
             const uint32_t hmask4 = rep4(0xFFu >> m);
+            const uint32_t half_off = first_of_pair ? 0 : 8;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-                const uint32_t h0 = (y[c].x >> m) & hmask4, h1 = (y[c].y >> m) & hmask4;
-                const uint32_t p0 = __shfl_down_sync(0xFFFFFFFFu, h0, pair_delta);
-                const uint32_t p1 = __shfl_down_sync(0xFFFFFFFFu, h1, pair_delta);
-                if (((wide_bits >> c) & 1) && first_of_pair && active) {
+                if (((wide_bits >> c) & 1) && active) {
                     const uint32_t grp = (c * n8 + j) >> 4;
                     const uint32_t rank = sh.prefix[grp >> 5] + __popc(sh.mask[grp >> 5] & ((1u << (grp & 31)) - 1));
-                    pack_record_any(hbits, make_uint4(h0, h1, p0, p1), smem_u32(s_rec) + rank * 2 * hbits);
+                    sts64(smem_u32(s_rec) + rank * 16 + half_off,
+                          make_uint2((y[c].x >> m) & hmask4, (y[c].y >> m) & hmask4));
                 }
             }
+        }
+    }
+    // Algorithm 2 over each wide group, one group per thread, packed in place: record i (2 hbits bytes)
+    // lands below the value bytes of every group that has not been read yet
+    if (N >= 128 && hbits > 0) {
+        __syncthreads();
+        for (uint32_t base = 0; base < wide_count; base += kEncodeThreads) {
+            const uint32_t i = base + tid;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (i < wide_count) v = lds128(smem_u32(s_rec) + i * 16);
+            __syncthreads();
+            if (i < wide_count) pack_record_any(hbits, v, smem_u32(s_rec) + i * 2 * hbits);
         }
     }
 
