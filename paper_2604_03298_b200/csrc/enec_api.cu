@@ -16,6 +16,7 @@ struct DeviceInfo {
     int sms = 0;
     bool decode_attr_set[2] = {false, false};
     bool hist_attr_set[2] = {false, false};
+    bool encode_attr_set[2] = {false, false};
 };
 
 static DeviceInfo& device_info(int dev) {
@@ -93,7 +94,15 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
         enec_histogram_kernel<DT><<<uint32_t(grid), kHistThreads, smem, stream>>>(job.in, job.count, job.ctl);
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
-    enec_encode_kernel<DT><<<nblocks, kEncodeThreads, 0, stream>>>(job, d_status);
+    if (!info.encode_attr_set[DT]) {
+        if (cudaFuncSetAttribute(enec_encode_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(EncodeSmem<DT>::kBytes)) != cudaSuccess)
+            return ENEC_ERR_CUDA;
+        info.encode_attr_set[DT] = true;
+    }
+    uint32_t grid = uint32_t(info.sms) * 4;  // four resident CTAs per SM, each takes block after block
+    if (grid > nblocks) grid = nblocks;
+    enec_encode_kernel<DT><<<grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream>>>(job, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }

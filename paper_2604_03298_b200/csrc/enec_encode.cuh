@@ -2,7 +2,7 @@
 //
 //   enec_histogram_kernel  Sec. 5.5 phase 1 (exponent histogram of the whole tensor) with the search of
 //                          phases 2 and 3 (Eq. 1, 3, 4) run by the last CTA to finish.
-//   enec_encode_kernel     one CTA per 16384-element block: split, transform (Eq. 2), group widths
+//   enec_encode_kernel     persistent CTAs, one 16384-element block at a time: split, transform (Eq. 2), group widths
 //                          (Sec. 5.2), Algorithm 2 on packed bytes for the low plane and for the records
 //                          of wide groups, and the block-offset prefix sum as a decoupled look-back over
 //                          per-block state words, so the input is read once.
@@ -30,10 +30,12 @@ struct alignas(16) EncodeControl {
 };
 static_assert(sizeof(EncodeControl) <= kControlBytes, "control area");
 
-// state word: bits 63..62 = kind, bits 31..0 = value
+// state word: bits 63..62 = kind, bit 61 = this block or one summed into the value saw parameters that lose
+// exponents, bits 31..0 = value. Failure travels inside the words, so no fence is needed around them.
 constexpr unsigned long long kStateAggregate = 1ull << 62;  // value = wide groups in the block
 constexpr unsigned long long kStatePrefix = 2ull << 62;     // value = wide groups up to and including the block
 constexpr unsigned long long kStatePoison = 3ull << 62;     // a predecessor failed
+constexpr unsigned long long kStateTaint = 1ull << 61;
 
 struct EncodeJob {
     const uint16_t* in;
@@ -478,10 +480,11 @@ struct EncodeShared {
     uint32_t mask[32];     // the block's group mask, bit g = group g is wide
     uint32_t prefix[32];   // wide groups before each mask word
     uint32_t group_or[8];  // short blocks: OR of y per group
-    uint32_t block;        // ticket
+    uint32_t next;         // ticket of the CTA's next block
     uint32_t wide;         // A_k
     uint32_t before;       // P_k
     uint32_t poisoned;
+    uint32_t tainted;      // the block or a predecessor saw parameters that lose exponents
 };
 
 // Phase 1 of a full block (16384 real elements), all 256 threads: loads, split, transform, sign/mantissa
@@ -614,37 +617,163 @@ __device__ __noinline__ int encode_short_block(const uint16_t* in, uint32_t N, u
     return bad;
 }
 
+// Dynamic shared memory of the encode kernel.
+template <int DT>
+struct EncodeSmem {
+    static constexpr uint32_t kHi3Bytes = DT == ENEC_FP16 ? kBlockElems * 3 / 8 : 32;
+    static constexpr uint32_t kBytes = kBlockElems + kHi3Bytes + 2 * kGroupsPerBlock * 16;
+};
+
+// What every block of the tensor shares.
+struct EncodeTensor {
+    Geometry g;
+    Sections sec;
+    int b, n, m, hbits;
+};
+
+// Second half of a block's work, all threads: find P_k (wide groups before block k) by looking back over
+// the predecessors' state words, publish the block's own prefix, copy its packed records (at shared
+// address `rec`, `wide_count` of them) to their place in the stream and write its table entry; the last
+// block also writes the header, the end of the table and the stream length. The look-back is done by
+// warp 0, up to 256 words per round trip, down to the nearest block that already knows its prefix.
+template <int DT>
+__device__ __forceinline__ void resolve_block(const EncodeJob& job, const EncodeTensor& t, uint32_t k, uint32_t wide_count,
+                                              bool own_taint, const uint8_t* rec, EncodeShared& sh, int* status) {
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (warp == 0 && k > 0) {
+        uint32_t before = 0;
+        uint32_t tainted = own_taint ? 1u : 0u;
+        int64_t pos = int64_t(k) - 1;
+        int outcome = 0;  // 1 = done, 2 = poisoned, 3 = gave up
+        uint32_t polls = 0;
+        while (outcome == 0) {
+            // eight coalesced loads of 32 consecutive words: word i * 32 + lane back from pos
+            unsigned long long st[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int64_t idx = pos - (i * 32 + int64_t(lane));
+                st[i] = idx >= 0 ? ld_relaxed_u64(&job.state[idx]) : kStatePrefix;
+            }
+            uint32_t mine = 0;      // this lane's share of the sum
+            uint32_t advanced = 0;  // windows of 32 fully summed in this round
+            bool blocked = false;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (outcome == 0 && !blocked) {
+                    const uint32_t kind = uint32_t(st[i] >> 62);
+                    const uint32_t prefix_lanes = __ballot_sync(0xFFFFFFFFu, kind == 2);
+                    const uint32_t empty_lanes = __ballot_sync(0xFFFFFFFFu, kind == 0);
+                    const uint32_t poison_lanes = __ballot_sync(0xFFFFFFFFu, kind == 3);
+                    const uint32_t first = prefix_lanes ? uint32_t(__ffs(prefix_lanes)) - 1 : 32;
+                    const uint32_t needed = first == 32 ? 0xFFFFFFFFu : (2u << first) - 1;  // lanes 0..first
+                    if (poison_lanes & needed) {
+                        outcome = 2;
+                    } else if (empty_lanes & needed) {
+                        blocked = true;  // a nearer block has not published yet
+                    } else {
+                        if ((needed >> lane) & 1) {
+                            mine += uint32_t(st[i]);
+                            tainted |= uint32_t(st[i] >> 61) & 1u;
+                        }
+                        if (first < 32) outcome = 1;
+                        else ++advanced;
+                    }
+                }
+            }
+            if (outcome == 2) break;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
+            before += mine;
+            pos -= 32 * int64_t(advanced);
+            if (blocked) {
+                if (++polls > (1u << 20)) { outcome = 3; break; }
+                __nanosleep(polls > 2 ? 400 : 100);
+            }
+        }
+        tainted = __any_sync(0xFFFFFFFFu, tainted != 0);
+        if (lane == 0) {
+            if (outcome == 1) {
+                sh.before = before;
+                sh.poisoned = 0;
+                sh.tainted = tainted;
+                st_relaxed_u64(&job.state[k], kStatePrefix | (tainted ? kStateTaint : 0ull) |
+                                                  (unsigned long long)(before + wide_count));
+            } else {
+                if (outcome == 3) report(status, ENEC_ERR_TIMEOUT);
+                st_relaxed_u64(&job.state[k], kStatePoison);
+                sh.poisoned = 1;
+                sh.tainted = 1;
+                sh.before = 0;
+            }
+        }
+    } else if (tid == 0 && k == 0) {
+        sh.before = 0;
+        sh.poisoned = 0;
+        sh.tainted = own_taint ? 1u : 0u;
+    }
+    __syncthreads();
+    const uint32_t before = sh.before;
+    const bool poisoned = sh.poisoned != 0;
+    const uint32_t hbits = uint32_t(t.hbits);
+    uint32_t* table = reinterpret_cast<uint32_t*>(job.out + t.sec.table);
+    if (!poisoned) {
+        // records to their place in the stream: record r of the tensor at r * 2 * hbits
+        uint16_t* dst = reinterpret_cast<uint16_t*>(job.out + t.sec.high + uint64_t(before) * 2 * hbits);
+        const uint16_t* src = reinterpret_cast<const uint16_t*>(rec);
+        for (uint32_t i = tid; i < wide_count * hbits; i += kEncodeThreads) dst[i] = src[i];
+        if (tid == 0) table[k] = before;
+    }
+    if (k + 1 == t.g.nblocks && tid == 0) {
+        const uint32_t a_total = before + wide_count;
+        const uint64_t high_bytes = uint64_t(a_total) * 2 * hbits;
+        const uint64_t total = t.sec.high + align16(high_bytes);
+        const bool failed = poisoned || sh.tainted != 0;
+        Header hd;
+        hd.magic = failed ? 0 : kMagic;
+        hd.version = kVersion;
+        hd.dtype = DT;
+        hd.pad0 = 0;
+        hd.count = job.count;
+        hd.block = kBlockElems;
+        hd.b = uint8_t(t.b); hd.n = uint8_t(t.n); hd.m = uint8_t(t.m); hd.L = kGroupElems;
+        hd.nblocks = t.g.nblocks;
+        hd.total_groups = t.g.total_groups;
+        hd.a_total = a_total;
+        hd.pad1 = 0;
+        hd.total_bytes = total;
+        hd.pad2[0] = hd.pad2[1] = 0;
+        *reinterpret_cast<Header*>(job.out) = hd;
+        if (!poisoned) {
+            table[t.g.nblocks] = a_total;
+            for (uint64_t i = uint64_t(t.g.nblocks) + 1; i < align16(4 * (uint64_t(t.g.nblocks) + 1)) / 4; ++i) table[i] = 0;
+            for (uint64_t p = high_bytes; p < align16(high_bytes); p += 2)
+                *reinterpret_cast<uint16_t*>(job.out + t.sec.high + p) = 0;
+        }
+        if (job.out_size) *job.out_size = failed ? 0ull : total;
+    }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kEncodeThreads, 4)
 enec_encode_kernel(EncodeJob job, int* status) {
     constexpr int E = DT == ENEC_BF16 ? 8 : 5;
-    __shared__ __align__(16) uint8_t s_low[kBlockElems];                              // normalised bytes, low plane
-    __shared__ __align__(16) uint8_t s_hi3[DT == ENEC_FP16 ? kBlockElems * 3 / 8 : 32];  // fp16 sign/mantissa-high plane
-    __shared__ __align__(16) uint8_t s_rec[kGroupsPerBlock * 16];  // wide groups in rank order: 16 value bytes, then packed
+    // dynamic shared memory: low plane | fp16 sign/mantissa-high plane | two record buffers
+    extern __shared__ __align__(16) uint8_t enc_smem[];
+    uint8_t* s_low = enc_smem;                                   // normalised bytes of the low plane
+    uint8_t* s_hi3 = enc_smem + kBlockElems;                     // fp16 only
+    uint8_t* s_rec_base = s_hi3 + EncodeSmem<DT>::kHi3Bytes;     // wide groups in rank order: 16 value bytes, then packed
     __shared__ EncodeShared sh;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) {
-        sh.block = atomicAdd(&job.ctl->ticket, 1u);
-        sh.poisoned = 0;
-    }
-    __syncthreads();
-    const uint32_t k = sh.block;
-
     int b = job.b, n = job.n, m = job.m;
     if (job.from_search) { b = job.ctl->b; n = job.ctl->n; m = job.ctl->m; }
     const int hbits = n - m;
-    const Geometry g = make_geometry(job.count);
-    const Sections sec = make_sections(DT, job.count, g, n, m, 0);
-    if (k >= g.nblocks) return;
-    const bool last = k + 1 == g.nblocks;
-    const uint32_t N = last ? g.tail_padded : kBlockElems;
-    const uint32_t real = last ? g.tail_real : kBlockElems;
-    const uint16_t* in = job.in + uint64_t(k) * kBlockElems;
-    uint8_t* out_sm = job.out + sec.sm + uint64_t(k) * kBlockElems;
-    uint8_t* out_low = job.out + sec.low + uint64_t(k) * (kBlockElems / 8) * uint32_t(m);
-    uint8_t* out_smhi = job.out + sec.smhi + uint64_t(k) * (kBlockElems / 8) * 3;
-    uint8_t* out_mask = job.out + sec.mask + uint64_t(k) * (kGroupsPerBlock / 8);
+    EncodeTensor tensor;
+    tensor.g = make_geometry(job.count);
+    tensor.sec = make_sections(DT, job.count, tensor.g, n, m, 0);
+    tensor.b = b; tensor.n = n; tensor.m = m; tensor.hbits = hbits;
+    const Geometry& g = tensor.g;
+    const Sections& sec = tensor.sec;
 
     TransformCtx tc;
     tc.b4 = rep4(uint32_t(b));
@@ -654,6 +783,30 @@ enec_encode_kernel(EncodeJob job, int* status) {
     tc.emask4 = rep4((1u << E) - 1);
     tc.n = n;
     tc.E = E;
+
+    // Persistent loop over tickets. A block's look-back is put off until the CTA has done the first half of
+    // its next block: by then the predecessors, which started at about the same time, have published their
+    // counts, so the wait that would otherwise hold the whole CTA is gone. Every count is published
+    // before its CTA waits for anything, and a wait only concerns blocks with smaller indices, so all
+    // waits end.
+    uint32_t pending_block = 0xFFFFFFFFu, pending_wide = 0, cur = 0;
+    bool pending_bad = false;
+    if (tid == 0) sh.next = atomicAdd(&job.ctl->ticket, 1u);
+    for (;;) {
+    __syncthreads();
+    const uint32_t k = sh.next;
+    if (k >= g.nblocks) break;
+    __syncthreads();  // everyone has read the ticket before the next one replaces it
+    if (tid == 0) sh.next = atomicAdd(&job.ctl->ticket, 1u);
+    uint8_t* s_rec = s_rec_base + cur * (kGroupsPerBlock * 16);
+    const bool last = k + 1 == g.nblocks;
+    const uint32_t N = last ? g.tail_padded : kBlockElems;
+    const uint32_t real = last ? g.tail_real : kBlockElems;
+    const uint16_t* in = job.in + uint64_t(k) * kBlockElems;
+    uint8_t* out_sm = job.out + sec.sm + uint64_t(k) * kBlockElems;
+    uint8_t* out_low = job.out + sec.low + uint64_t(k) * (kBlockElems / 8) * uint32_t(m);
+    uint8_t* out_smhi = job.out + sec.smhi + uint64_t(k) * (kBlockElems / 8) * 3;
+    uint8_t* out_mask = job.out + sec.mask + uint64_t(k) * (kGroupsPerBlock / 8);
 
     int bad = 0;
     uint2 y[8];
@@ -764,18 +917,14 @@ enec_encode_kernel(EncodeJob job, int* status) {
         sh.prefix[lane] = incl - __popc(mw);
         if (lane == 31) {
             sh.wide = incl;
-            if (any_bad) {
-                report(status, ENEC_ERR_PARAMS_NOT_LOSSLESS);
-                atomicOr(&job.ctl->error, 1u);
-            }
-            __threadfence();
+            if (any_bad) report(status, ENEC_ERR_PARAMS_NOT_LOSSLESS);
             // publish this block's count at once; block 0 knows its prefix already
-            st_relaxed_u64(&job.state[k], (k == 0 ? kStatePrefix : kStateAggregate) | incl);
+            st_relaxed_u64(&job.state[k], (k == 0 ? kStatePrefix : kStateAggregate) | (any_bad ? kStateTaint : 0ull) | incl);
+            if (k == 0) sh.before = 0;
         }
     }
     __syncthreads();
     const uint32_t wide_count = sh.wide;
-
     if (N >= 128) {
         fold_plane_out(smem_u32(s_low), N * uint32_t(m) / 8, out_low, tid);
         if (DT == ENEC_FP16) fold_plane_out(smem_u32(s_hi3), N * 3 / 8, out_smhi, tid);
@@ -811,92 +960,16 @@ enec_encode_kernel(EncodeJob job, int* status) {
         }
     }
 
-    // block-offset prefix sum: look back over the predecessors' state words (warp 0)
-    if (warp == 0 && k > 0) {
-        uint32_t before = 0;
-        int64_t pos = int64_t(k) - 1;
-        int outcome = 0;  // 1 = done, 2 = poisoned, 3 = gave up
-        uint32_t polls = 0;
-        while (outcome == 0) {
-            const int64_t idx = pos - lane;
-            unsigned long long st = idx >= 0 ? ld_relaxed_u64(&job.state[idx]) : kStatePrefix;
-            const uint32_t kind = uint32_t(st >> 62);
-            const uint32_t prefix_lanes = __ballot_sync(0xFFFFFFFFu, kind == 2);
-            const uint32_t empty_lanes = __ballot_sync(0xFFFFFFFFu, kind == 0);
-            const uint32_t poison_lanes = __ballot_sync(0xFFFFFFFFu, kind == 3);
-            const uint32_t first = prefix_lanes ? uint32_t(__ffs(prefix_lanes)) - 1 : 32;
-            const uint32_t needed = first == 32 ? 0xFFFFFFFFu : (2u << first) - 1;  // lanes 0..first
-            if (poison_lanes & needed) { outcome = 2; break; }
-            if (empty_lanes & needed) {
-                if (++polls > (1u << 20)) { outcome = 3; break; }
-                if (polls > 8) __nanosleep(200);
-                continue;
-            }
-            uint32_t v = (needed >> lane) & 1 ? uint32_t(st) : 0;
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-            before += v;
-            if (first < 32) outcome = 1;
-            else pos -= 32;
-        }
-        if (lane == 0) {
-            if (outcome == 1) {
-                sh.before = before;
-                __threadfence();
-                st_relaxed_u64(&job.state[k], kStatePrefix | (unsigned long long)(before + wide_count));
-            } else {
-                if (outcome == 3) report(status, ENEC_ERR_TIMEOUT);
-                atomicOr(&job.ctl->error, 1u);
-                __threadfence();
-                st_relaxed_u64(&job.state[k], kStatePoison);
-                sh.poisoned = 1;
-                sh.before = 0;
-            }
-        }
-    } else if (tid == 0 && k == 0) {
-        sh.before = 0;
+    // the previous block of this CTA, whose records wait in the other buffer
+    if (pending_block != 0xFFFFFFFFu)
+        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * (kGroupsPerBlock * 16), sh, status);
+    pending_block = k;
+    pending_wide = wide_count;
+    pending_bad = any_bad != 0;
+    cur ^= 1;
     }
-    __syncthreads();
-    const uint32_t before = sh.before;
-    const bool poisoned = sh.poisoned != 0;
-
-    uint32_t* table = reinterpret_cast<uint32_t*>(job.out + sec.table);
-    if (!poisoned) {
-        // records to their place in the stream: record r of the tensor at r * 2 * hbits
-        uint16_t* dst = reinterpret_cast<uint16_t*>(job.out + sec.high + uint64_t(before) * 2 * uint32_t(hbits));
-        const uint16_t* src = reinterpret_cast<const uint16_t*>(s_rec);
-        for (uint32_t i = tid; i < wide_count * uint32_t(hbits); i += kEncodeThreads) dst[i] = src[i];
-        if (tid == 0) table[k] = before;
-    }
-    if (last && tid == 0) {
-        const uint32_t a_total = before + wide_count;
-        const uint64_t high_bytes = uint64_t(a_total) * 2 * uint32_t(hbits);
-        const uint64_t total = sec.high + align16(high_bytes);
-        __threadfence();
-        const bool failed = poisoned || ld_relaxed_u32(&job.ctl->error) != 0;
-        Header hd;
-        hd.magic = failed ? 0 : kMagic;
-        hd.version = kVersion;
-        hd.dtype = DT;
-        hd.pad0 = 0;
-        hd.count = job.count;
-        hd.block = kBlockElems;
-        hd.b = uint8_t(b); hd.n = uint8_t(n); hd.m = uint8_t(m); hd.L = kGroupElems;
-        hd.nblocks = g.nblocks;
-        hd.total_groups = g.total_groups;
-        hd.a_total = a_total;
-        hd.pad1 = 0;
-        hd.total_bytes = total;
-        hd.pad2[0] = hd.pad2[1] = 0;
-        *reinterpret_cast<Header*>(job.out) = hd;
-        if (!poisoned) {
-            table[g.nblocks] = a_total;
-            for (uint64_t i = uint64_t(g.nblocks) + 1; i < align16(4 * (uint64_t(g.nblocks) + 1)) / 4; ++i) table[i] = 0;
-            for (uint64_t p = high_bytes; p < align16(high_bytes); p += 2)
-                *reinterpret_cast<uint16_t*>(job.out + sec.high + p) = 0;
-        }
-        if (job.out_size) *job.out_size = failed ? 0ull : total;
-    }
+    if (pending_block != 0xFFFFFFFFu)
+        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * (kGroupsPerBlock * 16), sh, status);
 }
 
 // Stream of an empty tensor: header and a one-entry table.
