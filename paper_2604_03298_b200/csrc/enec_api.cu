@@ -28,6 +28,24 @@ static DeviceInfo& device_info(int dev) {
     return d;
 }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
+// stream drains; it waits for the predecessor's completion itself (pdl_wait) before touching memory.
+template <class... KernelArgs, class... Args>
+static cudaError_t launch_pdl(void (*kernel)(KernelArgs...), uint32_t grid, uint32_t threads, size_t smem,
+                              cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KernelArgs(args)...);
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 template <int DT>
@@ -44,9 +62,9 @@ static enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaSt
     uint32_t grid = uint32_t(info.sms) * 3;  // three resident CTAs per SM
     if (grid > batch.total_blocks) grid = batch.total_blocks;
     if (grid == 0) grid = 1;
-    enec_decode_kernel<DT><<<grid, kDecodeThreads, kDecodeSmemBytes, stream>>>(batch, d_status);
+    const cudaError_t err = launch_pdl(enec_decode_kernel<DT>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
+    return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
 
 // Device scratch, one area per (device, stream, purpose): for the compressor control words and one state
@@ -91,7 +109,9 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
         uint64_t grid = (chunks + kHistThreads - 1) / kHistThreads;
         if (grid > uint64_t(info.sms) * 3) grid = uint64_t(info.sms) * 3;
         if (grid == 0) grid = 1;
-        enec_histogram_kernel<DT><<<uint32_t(grid), kHistThreads, smem, stream>>>(job.in, job.count, job.ctl);
+        if (launch_pdl(enec_histogram_kernel<DT>, uint32_t(grid), kHistThreads, smem, stream, job.in, job.count,
+                       job.ctl) != cudaSuccess)
+            return ENEC_ERR_CUDA;
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
     if (!info.encode_attr_set[DT]) {
@@ -102,9 +122,9 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
     }
     uint32_t grid = uint32_t(info.sms) * 4;  // four resident CTAs per SM, each takes block after block
     if (grid > nblocks) grid = nblocks;
-    enec_encode_kernel<DT><<<grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream>>>(job, d_status);
+    const cudaError_t err = launch_pdl(enec_encode_kernel<DT>, grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream, job, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
+    return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
 
 static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count, bool with_params, int b, int n,

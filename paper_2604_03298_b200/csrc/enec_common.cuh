@@ -184,6 +184,14 @@ __host__ __device__ constexpr int bitrev(int t, int f) {
     return r;
 }
 
+// Programmatic dependent launch. A kernel launched with programmatic stream serialisation may start
+// while the kernel before it in the stream is still running: pdl_wait() blocks until that kernel has
+// finished and its memory is visible (it returns at once under an ordinary launch); everything that
+// touches global memory comes after it. pdl_launch_dependents() lets the next kernel of the stream be
+// scheduled into SM resources as they free up, so its launch latency hides behind this kernel's tail.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void report(int* status, int code) {
     if (status) atomicCAS(status, 0, code);
 }

@@ -562,6 +562,8 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
     const uint32_t stages = smem_u32(smem) + uint32_t(sizeof(DecodeShared));
     constexpr uint32_t S = kStages;
 
+    pdl_launch_dependents();
+    pdl_wait();  // nothing above touches global memory
     if (batch.total_blocks == 0) {  // nothing to decode: only check the header of a single empty tensor
         if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr) {
             JobCtx jc;

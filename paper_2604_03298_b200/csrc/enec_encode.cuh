@@ -214,6 +214,8 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     __shared__ uint32_t cta_hist[256];
     __shared__ int s_last;
     constexpr int kWarpBytes = HistShape<DT>::kWarpBytes;
+    pdl_launch_dependents();
+    pdl_wait();  // nothing above touches global memory
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t warp_base = smem_u32(smem) + warp * kWarpBytes;
     const uint32_t base = warp_base + lane * 4;
@@ -764,6 +766,8 @@ enec_encode_kernel(EncodeJob job, int* status) {
     uint8_t* s_rec_base = s_hi3 + EncodeSmem<DT>::kHi3Bytes;     // wide groups in rank order: 16 value bytes, then packed
     __shared__ EncodeShared sh;
 
+    pdl_launch_dependents();
+    pdl_wait();  // nothing above touches global memory
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int b = job.b, n = job.n, m = job.m;
     if (job.from_search) { b = job.ctl->b; n = job.ctl->n; m = job.ctl->m; }
