@@ -363,59 +363,76 @@ template <int DT, int M, int HB>
 __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_low, uint32_t s_smhi, uint32_t tid) {
     constexpr int n = M + HB;
     constexpr uint32_t Hm = 0x80808080u;
-    uint2 y[8];
-    uint2 hs[8];
-    unpack_plane<M>(s_low, 8 * tid, kBlockElems, y);
-    if (DT == ENEC_FP16) unpack_plane<3>(s_smhi, 8 * tid, kBlockElems, hs);
     const uint32_t rank_addr = r.rank + (tid >> 1) * 2;
     const uint32_t exp_addr = r.expanded + (tid & 1) * 8;
     const uint32_t sm_addr = r.sm + 8 * tid;
     uint4* out = reinterpret_cast<uint4*>(r.out + 8 * tid);
+    // Shared-memory loads are issued in batches ahead of the arithmetic that uses them (the load helpers
+    // keep program order): all rank entries first, then the planes, then per half of the runs the
+    // expanded high bits and the sign/mantissa bytes.
+    uint32_t rk[8];
+    if constexpr (HB > 0) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint2 v = y[c];
+        for (int c = 0; c < 8; ++c) rk[c] = lds16(rank_addr + c * (kBlockElems / 8 / 16) * 2);
+    }
+    uint2 y[8];
+    uint2 hs[8];
+    unpack_plane<M>(s_low, 8 * tid, kBlockElems, y);
+    if (DT == ENEC_FP16) unpack_plane<3>(s_smhi, 8 * tid, kBlockElems, hs);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint2 hi[4];
+        uint2 smv[4];
         if constexpr (HB > 0) {
-            const uint32_t rk = lds16(rank_addr + c * (kBlockElems / 8 / 16) * 2);
-            const uint2 hi = lds64(exp_addr + rk * 16);
-            v.x += hi.x << M;  // disjoint bits
-            v.y += hi.y << M;
-        } else {
-            v.x ^= r.s4;
-            v.y ^= r.s4;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) hi[q] = lds64(exp_addr + rk[4 * h + q] * 16);
         }
-        uint32_t x0, x1;
-        if constexpr (DT == ENEC_FP16) {
-            // b + 2^(n-1) < 128: the guard bit absorbs any borrow and is masked away with the field
-            x0 = r.c4_or_h - v.x;
-            x1 = r.c4_or_h - v.y;
-        } else if constexpr (n < 8) {
-            x0 = r.c4 - v.x;
-            x1 = r.c4 - v.y;
-        } else {  // n = 8: bytewise (b + 128) - (y ^ 128) modulo 256
-            x0 = (r.c4_or_h - (v.x & ~Hm)) ^ ((r.c4 ^ ~v.x) & Hm);
-            x1 = (r.c4_or_h - (v.y & ~Hm)) ^ ((r.c4 ^ ~v.y) & Hm);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) smv[q] = lds64(sm_addr + (4 * h + q) * (kBlockElems / 8));
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int c = 4 * h + q;
+            uint2 v = y[c];
+            if constexpr (HB > 0) {
+                v.x += hi[q].x << M;  // disjoint bits
+                v.y += hi[q].y << M;
+            } else {
+                v.x ^= r.s4;
+                v.y ^= r.s4;
+            }
+            uint32_t x0, x1;
+            if constexpr (DT == ENEC_FP16) {
+                // b + 2^(n-1) < 128: the guard bit absorbs any borrow and is masked away with the field
+                x0 = r.c4_or_h - v.x;
+                x1 = r.c4_or_h - v.y;
+            } else if constexpr (n < 8) {
+                x0 = r.c4 - v.x;
+                x1 = r.c4 - v.y;
+            } else {  // n = 8: bytewise (b + 128) - (y ^ 128) modulo 256
+                x0 = (r.c4_or_h - (v.x & ~Hm)) ^ ((r.c4 ^ ~v.x) & Hm);
+                x1 = (r.c4_or_h - (v.y & ~Hm)) ^ ((r.c4 ^ ~v.y) & Hm);
+            }
+            uint32_t lo0, lo1, hi0, hi1;
+            if (DT == ENEC_BF16) {
+                hi0 = (smv[q].x & Hm) | ((x0 >> 1) & ~Hm);
+                hi1 = (smv[q].y & Hm) | ((x1 >> 1) & ~Hm);
+                lo0 = ((x0 << 7) & Hm) | (smv[q].x & ~Hm);
+                lo1 = ((x1 << 7) & Hm) | (smv[q].y & ~Hm);
+            } else {
+                x0 &= 0x1F1F1F1Fu;
+                x1 &= 0x1F1F1F1Fu;
+                hi0 = ((hs[c].x << 5) & Hm) | (x0 << 2) | (hs[c].x & 0x03030303u);
+                hi1 = ((hs[c].y << 5) & Hm) | (x1 << 2) | (hs[c].y & 0x03030303u);
+                lo0 = smv[q].x;
+                lo1 = smv[q].y;
+            }
+            uint4 w;
+            w.x = prmt(lo0, hi0, 0x5140u);
+            w.y = prmt(lo0, hi0, 0x7362u);
+            w.z = prmt(lo1, hi1, 0x5140u);
+            w.w = prmt(lo1, hi1, 0x7362u);
+            out[c * (kBlockElems / 8 / 8)] = w;
         }
-        const uint2 smv = lds64(sm_addr + c * (kBlockElems / 8));
-        uint32_t lo0, lo1, hi0, hi1;
-        if (DT == ENEC_BF16) {
-            hi0 = (smv.x & Hm) | ((x0 >> 1) & ~Hm);
-            hi1 = (smv.y & Hm) | ((x1 >> 1) & ~Hm);
-            lo0 = ((x0 << 7) & Hm) | (smv.x & ~Hm);
-            lo1 = ((x1 << 7) & Hm) | (smv.y & ~Hm);
-        } else {
-            x0 &= 0x1F1F1F1Fu;
-            x1 &= 0x1F1F1F1Fu;
-            hi0 = ((hs[c].x << 5) & Hm) | (x0 << 2) | (hs[c].x & 0x03030303u);
-            hi1 = ((hs[c].y << 5) & Hm) | (x1 << 2) | (hs[c].y & 0x03030303u);
-            lo0 = smv.x;
-            lo1 = smv.y;
-        }
-        uint4 w;
-        w.x = prmt(lo0, hi0, 0x5140u);
-        w.y = prmt(lo0, hi0, 0x7362u);
-        w.z = prmt(lo1, hi1, 0x5140u);
-        w.w = prmt(lo1, hi1, 0x7362u);
-        out[c * (kBlockElems / 8 / 8)] = w;
     }
 }
 
@@ -623,7 +640,17 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
             const uint32_t k = gb - job_first;
             uint32_t t0;
             if (!parsed) {
-                const int err = load_job<DT>(batch.jobs ? batch.jobs[j] : batch.single, jc);
+                const DecodeJob job = batch.jobs ? batch.jobs[j] : batch.single;
+                // the table sits right behind the header: fetch the block's two entries along with the
+                // header instead of after it (they are only used once the header has been checked)
+                uint32_t e0 = 0, e1 = 0;
+                const bool early = job.in_size >= kHeaderBytes + 4 * (uint64_t(k) + 2);
+                if (early) {
+                    const uint32_t* tb = reinterpret_cast<const uint32_t*>(job.in + kHeaderBytes);
+                    e0 = tb[k];
+                    e1 = tb[k + 1];
+                }
+                const int err = early ? load_job<DT>(job, jc) : ENEC_ERR_BAD_STREAM;
                 if (err) {
                     *abort_flag = 1;
                     report(status, err);
@@ -633,8 +660,8 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
                 hbits = jc.n - jc.m;
                 L = make_stage_layout(DT, jc.m, hbits);
                 table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
-                t0 = table[k];
-                t1 = table[k + 1];
+                t0 = e0;
+                t1 = e1;
                 parsed = true;
             } else {
                 t0 = t1;
