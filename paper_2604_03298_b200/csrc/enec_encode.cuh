@@ -623,7 +623,8 @@ __device__ __noinline__ int encode_short_block(const uint16_t* in, uint32_t N, u
 template <int DT>
 struct EncodeSmem {
     static constexpr uint32_t kHi3Bytes = DT == ENEC_FP16 ? kBlockElems * 3 / 8 : 32;
-    static constexpr uint32_t kBytes = kBlockElems + kHi3Bytes + 2 * kGroupsPerBlock * 16;
+    static constexpr uint32_t kRecBytes = kGroupsPerBlock * 16 + 16;  // one buffer: every group wide, plus a spare slot
+    static constexpr uint32_t kBytes = kBlockElems + kHi3Bytes + 2 * kRecBytes;
 };
 
 // What every block of the tensor shares.
@@ -802,7 +803,7 @@ enec_encode_kernel(EncodeJob job, int* status) {
     if (k >= g.nblocks) break;
     __syncthreads();  // everyone has read the ticket before the next one replaces it
     if (tid == 0) sh.next = atomicAdd(&job.ctl->ticket, 1u);
-    uint8_t* s_rec = s_rec_base + cur * (kGroupsPerBlock * 16);
+    uint8_t* s_rec = s_rec_base + cur * EncodeSmem<DT>::kRecBytes;
     const bool last = k + 1 == g.nblocks;
     const uint32_t N = last ? g.tail_padded : kBlockElems;
     const uint32_t real = last ? g.tail_real : kBlockElems;
@@ -908,6 +909,16 @@ enec_encode_kernel(EncodeJob job, int* status) {
                                      reinterpret_cast<uint32_t*>(s_rec));
     }
     const int any_bad = __syncthreads_or(bad);
+    {
+        // the CTA's next block is known by now: pull its 32 KB towards L2 (one 128-byte line per thread)
+        // so that the loads of the next iteration do not wait for DRAM
+        const uint32_t next_block = sh.next;
+        if (next_block < g.nblocks) {
+            const uint8_t* line = reinterpret_cast<const uint8_t*>(job.in + uint64_t(next_block) * kBlockElems) + tid * 128;
+            const uint8_t* end = reinterpret_cast<const uint8_t*>(job.in + job.count);
+            if (line < end) asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
+        }
+    }
 
     // wide groups before each mask word, and in the block
     if (warp == 0) {
@@ -935,19 +946,20 @@ enec_encode_kernel(EncodeJob job, int* status) {
         const uint32_t mask_vecs = uint32_t(align16(((N >> 4) + 7) / 8)) / 16;
         if (tid < mask_vecs)
             reinterpret_cast<uint4*>(out_mask)[tid] = reinterpret_cast<const uint4*>(sh.mask)[tid];
-        // high bits of wide groups into shared memory, rank order, sixteen value bytes per group:
-        // each lane of a pair stores its own half
+        // high bits of wide groups into shared memory, rank order, sixteen value bytes per group: each
+        // lane of a pair stores its own half; narrow groups store to a spare slot behind the buffer, so
+        // there is no branch
         if (hbits > 0) {
             const uint32_t hmask4 = rep4(0xFFu >> m);
             const uint32_t half_off = first_of_pair ? 0 : 8;
+            const uint32_t spare = kGroupsPerBlock * 16;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-                if (((wide_bits >> c) & 1) && active) {
-                    const uint32_t grp = (c * n8 + j) >> 4;
-                    const uint32_t rank = sh.prefix[grp >> 5] + __popc(sh.mask[grp >> 5] & ((1u << (grp & 31)) - 1));
-                    sts64(smem_u32(s_rec) + rank * 16 + half_off,
-                          make_uint2((y[c].x >> m) & hmask4, (y[c].y >> m) & hmask4));
-                }
+                const uint32_t grp = (c * n8 + j) >> 4;
+                const uint32_t rank = sh.prefix[(grp >> 5) & 31] + __popc(sh.mask[(grp >> 5) & 31] & ((1u << (grp & 31)) - 1));
+                const bool wide = ((wide_bits >> c) & 1) && active;
+                sts64(smem_u32(s_rec) + (wide ? rank * 16 : spare) + half_off,
+                      make_uint2((y[c].x >> m) & hmask4, (y[c].y >> m) & hmask4));
             }
         }
     }
@@ -966,14 +978,14 @@ enec_encode_kernel(EncodeJob job, int* status) {
 
     // the previous block of this CTA, whose records wait in the other buffer
     if (pending_block != 0xFFFFFFFFu)
-        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * (kGroupsPerBlock * 16), sh, status);
+        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
     pending_block = k;
     pending_wide = wide_count;
     pending_bad = any_bad != 0;
     cur ^= 1;
     }
     if (pending_block != 0xFFFFFFFFu)
-        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * (kGroupsPerBlock * 16), sh, status);
+        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
 }
 
 // Stream of an empty tensor: header and a one-entry table.
