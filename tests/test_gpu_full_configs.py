@@ -80,3 +80,50 @@ def test_config5_moe_full(oracle):
     reuse = lambda i, s: (s.shape, i % 24) if len(s.shape) == 2 else ("v", i)
     ratio = _run_set(specs, oracle, sample=(0, 1, 2, 767, 768, 769, 2000, 4863), reuse=reuse)
     assert 1.36 < ratio < 1.40
+
+
+def test_tensor_beyond_four_gigabytes():
+    """2^31 + 49157 bf16 values (4.3 GB): byte offsets pass 2^32 and block counts pass 2^17, the tail is ragged.
+    The oracle would need minutes for this, so the checks are the ones that hold at any size: bit-exact round trip,
+    header fields, and the stream length rebuilt from the table's last entry by the closed form of the layout."""
+    import paper_2604_03298_b200 as enec
+    count = (1 << 31) + 49157
+    g = torch.Generator(device="cuda").manual_seed(77)
+    t = torch.empty(count, dtype=torch.bfloat16, device="cuda")
+    step = 1 << 28
+    for lo in range(0, count, step):
+        hi = min(count, lo + step)
+        x = torch.randn(hi - lo, generator=g, device="cuda", dtype=torch.float32)
+        x = torch.where(x == 0, torch.full_like(x, 2.0 ** -10), x) * 0.02
+        t[lo:hi] = x.to(torch.bfloat16)
+        del x
+    cap = enec.enec_max_compressed_size(0, count)
+    buf = torch.empty(cap, dtype=torch.uint8, device="cuda")
+    size = torch.zeros(1, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert enec.enec_compress(t, 0, count, buf, cap, size, status) == 0
+    out = torch.empty_like(t)
+    assert enec.enec_decompress(buf, cap, 0, count, out, status) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for lo in range(0, count, step):      # chunked compare keeps the temporaries small
+        hi = min(count, lo + step)
+        assert torch.equal(out[lo:hi].view(torch.int16), t[lo:hi].view(torch.int16))
+    n = int(size.item())
+    head = buf[:64].cpu().numpy()
+    nblocks = (count + 16383) // 16384
+    assert int(head[8:16].view(np.uint64)[0]) == count
+    assert int(head[24:28].view(np.uint32)[0]) == nblocks
+    b, nn, m = int(head[20]), int(head[21]), int(head[22])
+    assert (nn, m) == (6, 3) and 119 <= b <= 123
+    a_total = int(head[32:36].view(np.uint32)[0])
+    table_last = int(buf[64 + 4 * nblocks:64 + 4 * nblocks + 4].cpu().numpy().view(np.uint32)[0])
+    assert table_last == a_total
+    a16 = lambda v: (v + 15) // 16 * 16
+    tail_real = count - (nblocks - 1) * 16384
+    tail_pad = 16
+    while tail_pad < tail_real:
+        tail_pad *= 2
+    padded = (nblocks - 1) * 16384 + tail_pad
+    expect = 64 + a16(4 * (nblocks + 1)) + a16((padded // 16 + 7) // 8) + a16(padded * m // 8) + a16(count) + a16(a_total * 2 * (nn - m))
+    assert n == expect == int(head[40:48].view(np.uint64)[0])
