@@ -25,7 +25,7 @@ struct alignas(16) EncodeControl {
     unsigned long long hist[256];  // exponent histogram (2^E bins used)
     uint32_t ticket;               // next block to hand out
     uint32_t hist_done;            // CTAs of the histogram kernel that have finished
-    uint32_t error;                // some block failed; the header is not written
+    uint32_t reserved;
     int b, n, m;                   // result of the parameter search
 };
 static_assert(sizeof(EncodeControl) <= kControlBytes, "control area");
@@ -87,12 +87,18 @@ __device__ __forceinline__ uint32_t counter_offset(uint32_t x) {
 
 template <int DT>
 __device__ __forceinline__ void count_word_pair(uint32_t base, uint32_t w) {
-    // two 16-bit values per 32-bit word
-    constexpr int sh = DT == ENEC_BF16 ? 7 : 10;
-    constexpr uint32_t fm = DT == ENEC_BF16 ? 0xFFu : 0x1Fu;
-    const uint32_t a0 = base + counter_offset<DT>((w >> sh) & fm);
+    // two 16-bit values per 32-bit word; the counter's offset is taken straight from the word's bits
+    uint32_t a0, a1;
+    if (DT == ENEC_BF16) {
+        // exponent x = bits 14..7: offset = (x & 63) << 7 | x >> 6 = (w & 0x1F80) + (bits 14..13)
+        a0 = base + (w & 0x1F80u) + ((w >> 13) & 3u);
+        a1 = base + ((w >> 16) & 0x1F80u) + ((w >> 29) & 3u);
+    } else {
+        // exponent x = bits 14..10: offset = (x & 7) << 7 | x >> 3
+        a0 = base + ((w >> 3) & 0x380u) + ((w >> 13) & 3u);
+        a1 = base + ((w >> 19) & 0x380u) + ((w >> 29) & 3u);
+    }
     sts8(a0, lds8(a0) + 1);
-    const uint32_t a1 = base + counter_offset<DT>((w >> (16 + sh)) & fm);
     sts8(a1, lds8(a1) + 1);
 }
 
