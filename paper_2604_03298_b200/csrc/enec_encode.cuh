@@ -486,10 +486,8 @@ __device__ __forceinline__ uint32_t lossy_bytes(const TransformCtx& t, uint32_t 
 // ---------------------------------------------------------------------------------------------------
 struct EncodeShared {
     uint32_t mask[32];     // the block's group mask, bit g = group g is wide
-    uint32_t prefix[32];   // wide groups before each mask word
     uint32_t group_or[8];  // short blocks: OR of y per group
-    uint32_t next;         // ticket of the CTA's next block
-    uint32_t wide;         // A_k
+    uint32_t next[2];      // tickets of the CTA's current and next block, by iteration parity
     uint32_t before;       // P_k
     uint32_t poisoned;
     uint32_t tainted;      // the block or a predecessor saw parameters that lose exponents
@@ -802,13 +800,13 @@ enec_encode_kernel(EncodeJob job, int* status) {
     // waits end.
     uint32_t pending_block = 0xFFFFFFFFu, pending_wide = 0, cur = 0;
     bool pending_bad = false;
-    if (tid == 0) sh.next = atomicAdd(&job.ctl->ticket, 1u);
-    for (;;) {
+    if (tid == 0) sh.next[0] = atomicAdd(&job.ctl->ticket, 1u);
+    for (uint32_t iter = 0;; ++iter) {
     __syncthreads();
-    const uint32_t k = sh.next;
+    const uint32_t k = sh.next[iter & 1];
     if (k >= g.nblocks) break;
-    __syncthreads();  // everyone has read the ticket before the next one replaces it
-    if (tid == 0) sh.next = atomicAdd(&job.ctl->ticket, 1u);
+    // the ticket after this one goes to the other slot, which nobody reads before the next barrier
+    if (tid == 0) sh.next[(iter + 1) & 1] = atomicAdd(&job.ctl->ticket, 1u);
     uint8_t* s_rec = s_rec_base + cur * EncodeSmem<DT>::kRecBytes;
     const bool last = k + 1 == g.nblocks;
     const uint32_t N = last ? g.tail_padded : kBlockElems;
@@ -918,7 +916,7 @@ enec_encode_kernel(EncodeJob job, int* status) {
     {
         // the CTA's next block is known by now: pull its 32 KB towards L2 (one 128-byte line per thread)
         // so that the loads of the next iteration do not wait for DRAM
-        const uint32_t next_block = sh.next;
+        const uint32_t next_block = sh.next[(iter + 1) & 1];
         if (next_block < g.nblocks) {
             const uint8_t* line = reinterpret_cast<const uint8_t*>(job.in + uint64_t(next_block) * kBlockElems) + tid * 128;
             const uint8_t* end = reinterpret_cast<const uint8_t*>(job.in + job.count);
@@ -926,26 +924,22 @@ enec_encode_kernel(EncodeJob job, int* status) {
         }
     }
 
-    // wide groups before each mask word, and in the block
-    if (warp == 0) {
-        const uint32_t mw = sh.mask[lane];
-        uint32_t incl = __popc(mw);
+    // wide groups before each mask word and in the block: every warp scans the 32 mask words itself
+    // (lane l holds word l), so no second barrier is needed
+    const uint32_t mask_word = sh.mask[lane];
+    uint32_t mask_incl = __popc(mask_word);
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-            if (lane >= uint32_t(d)) incl += t;
-        }
-        sh.prefix[lane] = incl - __popc(mw);
-        if (lane == 31) {
-            sh.wide = incl;
-            if (any_bad) report(status, ENEC_ERR_PARAMS_NOT_LOSSLESS);
-            // publish this block's count at once; block 0 knows its prefix already
-            st_relaxed_u64(&job.state[k], (k == 0 ? kStatePrefix : kStateAggregate) | (any_bad ? kStateTaint : 0ull) | incl);
-            if (k == 0) sh.before = 0;
-        }
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, mask_incl, d);
+        if (lane >= uint32_t(d)) mask_incl += t;
     }
-    __syncthreads();
-    const uint32_t wide_count = sh.wide;
+    const uint32_t mask_excl = mask_incl - __popc(mask_word);
+    const uint32_t wide_count = __shfl_sync(0xFFFFFFFFu, mask_incl, 31);
+    if (tid == 31) {
+        if (any_bad) report(status, ENEC_ERR_PARAMS_NOT_LOSSLESS);
+        // publish this block's count at once; block 0 knows its prefix already
+        st_relaxed_u64(&job.state[k], (k == 0 ? kStatePrefix : kStateAggregate) | (any_bad ? kStateTaint : 0ull) | wide_count);
+    }
     if (N >= 128) {
         fold_plane_out(smem_u32(s_low), N * uint32_t(m) / 8, out_low, tid);
         if (DT == ENEC_FP16) fold_plane_out(smem_u32(s_hi3), N * 3 / 8, out_smhi, tid);
@@ -962,7 +956,9 @@ enec_encode_kernel(EncodeJob job, int* status) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const uint32_t grp = (c * n8 + j) >> 4;
-                const uint32_t rank = sh.prefix[(grp >> 5) & 31] + __popc(sh.mask[(grp >> 5) & 31] & ((1u << (grp & 31)) - 1));
+                const uint32_t word = (grp >> 5) & 31;
+                const uint32_t rank = __shfl_sync(0xFFFFFFFFu, mask_excl, word) +
+                                      __popc(__shfl_sync(0xFFFFFFFFu, mask_word, word) & ((1u << (grp & 31)) - 1));
                 const bool wide = ((wide_bits >> c) & 1) && active;
                 sts64(smem_u32(s_rec) + (wide ? rank * 16 : spare) + half_off,
                       make_uint2((y[c].x >> m) & hmask4, (y[c].y >> m) & hmask4));
