@@ -243,7 +243,9 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
         for (uint32_t u = 0; u < kUnroll; ++u) {
             const uint64_t i = first + u * 32 + lane;
             v[u] = make_uint4(0, 0, 0, 0);
-            if (i < nchunks) v[u] = in4[i];  // default caching: the encode pass reads the tensor again
+            // back to front, default caching: the encode pass reads the tensor again from the front, where
+            // the lines touched last are the likeliest to be in L2 still
+            if (i < nchunks) v[u] = in4[nchunks - 1 - i];
         }
 #pragma unroll
         for (uint32_t u = 0; u < kUnroll; ++u) {
