@@ -535,6 +535,24 @@ static_assert(sizeof(DecodeShared) == 128, "control area is 128 bytes");
     X(DT, 7, 0) X(DT, 7, 1)                                                                           \
     X(DT, 8, 0)
 
+// Bounded wait of any number of threads: each try suspends the thread for up to 20 us or until the phase
+// completes, and there are at most 2^16 tries (about a second); also gives up when the CTA aborts.
+__device__ __forceinline__ bool suspended_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < (1u << 16); ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
+            : "memory");
+        if (ok) return true;
+        if (*abort_flag) return false;
+    }
+    return false;
+}
+
 // Bounded wait by one thread; also gives up when the CTA aborts. Sleeps between polls so that a waiting
 // thread leaves the issue slots to the warps that have work.
 __device__ __forceinline__ bool poll_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -724,15 +742,14 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
     for (uint32_t i = 0; i < n_mine; ++i) {
         const uint32_t s = i % S, use = i / S;
         const uint32_t st = stages + s * kStageBytes;
-        // one thread waits for the block's bytes; the others sleep at the barrier
-        bool failed = false;
-        if (tid == 0 && !poll_wait(&ctl->full[s], use & 1, abort_flag)) {
-            failed = true;
-            if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
+        // every consumer thread waits on the stage's mbarrier itself; the wait suspends the thread in hardware,
+        // so waiting threads take no issue slots and wake the moment the copies have landed
+        const bool arrived = suspended_wait(&ctl->full[s], use & 1, abort_flag);
+        if (__any_sync(0xFFFFFFFFu, !arrived)) {
+            if (lane == 0 && !*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
+            consumer_barrier_or(true);  // the block's one barrier: the other warps leave with this one
+            break;
         }
-        // every consumer reaches both barriers of a block, failed wait or not, and all leave together
-        if (consumer_barrier_or(failed || *abort_flag != 0)) break;
-        mbar_try_wait(&ctl->full[s], use & 1);  // completed: acquires the copied bytes in every thread
         const BlockDesc* d = reinterpret_cast<const BlockDesc*>(smem + sizeof(DecodeShared) + size_t(s) * kStageBytes);
         const uint32_t N = d->N, expect = d->expect, code = d->code;
         const uint32_t b = d->b, n = d->n;
