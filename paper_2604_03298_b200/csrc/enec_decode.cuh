@@ -553,17 +553,6 @@ __device__ __forceinline__ bool suspended_wait(uint64_t* bar, uint32_t parity, v
     return false;
 }
 
-// Bounded wait by one thread; also gives up when the CTA aborts. Sleeps between polls so that a waiting
-// thread leaves the issue slots to the warps that have work.
-__device__ __forceinline__ bool poll_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        __nanosleep(it < 64 ? 32 : 256);
-    }
-    return false;
-}
-
 // What the loader tells the consumers about the block in a stage (first bytes of the stage).
 struct BlockDesc {
     uint32_t first;     // offset of the block's first record inside the staged window
@@ -686,7 +675,7 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
                 t1 = t2;
             }
             const uint32_t s = issued % S, use = issued / S;
-            if (use > 0 && !poll_wait(&ctl->empty[s], (use - 1) & 1, abort_flag)) { failed = true; break; }
+            if (use > 0 && !suspended_wait(&ctl->empty[s], (use - 1) & 1, abort_flag)) { failed = true; break; }
             const bool tail = (k + 1 == jc.nblocks);
             const uint32_t N = tail ? jc.tail_padded : kBlockElems;
             const uint32_t real = tail ? jc.tail_real : kBlockElems;
