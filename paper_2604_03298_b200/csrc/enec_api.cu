@@ -221,8 +221,10 @@ enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, siz
     batch.prefix = nullptr;
     batch.n_jobs = 1;
     batch.total_blocks = make_geometry(count).nblocks;
-    batch.single = DecodeJob{static_cast<const uint8_t*>(d_in), static_cast<uint16_t*>(d_out), uint64_t(count),
-                             uint64_t(in_size)};
+    batch.inline_jobs[0] = DecodeJob{static_cast<const uint8_t*>(d_in), static_cast<uint16_t*>(d_out), uint64_t(count),
+                                     uint64_t(in_size)};
+    batch.inline_prefix[0] = 0;
+    batch.inline_prefix[1] = batch.total_blocks;
     return dt == ENEC_BF16 ? launch_decode<ENEC_BF16>(batch, d_status, stream)
                            : launch_decode<ENEC_FP16>(batch, d_status, stream);
 }
@@ -253,20 +255,27 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
     }
     prefix[n_items] = uint32_t(total);
     if (total == 0) return ENEC_OK;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
-    uint8_t* scratch = nullptr;
-    const enec_status st = get_scratch(dev, stream, kScratchBatch, host.size(), &scratch);
-    if (st != ENEC_OK) return st;
-    // pageable source: the call returns once the bytes are staged, so `host` may go out of scope
-    if (cudaMemcpyAsync(scratch, host.data(), host.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
-        return ENEC_ERR_CUDA;
     DecodeBatch batch;
-    batch.jobs = reinterpret_cast<const DecodeJob*>(scratch);
-    batch.prefix = reinterpret_cast<const uint32_t*>(scratch + jobs_bytes);
     batch.n_jobs = uint32_t(n_items);
     batch.total_blocks = uint32_t(total);
-    batch.single = DecodeJob{nullptr, nullptr, 0, 0};
+    if (uint32_t(n_items) <= kInlineJobs) {
+        // a short list travels in the launch parameters: no copy, no scratch
+        batch.jobs = nullptr;
+        batch.prefix = nullptr;
+        for (int i = 0; i < n_items; ++i) batch.inline_jobs[i] = jobs[i];
+        for (int i = 0; i <= n_items; ++i) batch.inline_prefix[i] = prefix[i];
+    } else {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
+        uint8_t* scratch = nullptr;
+        const enec_status st = get_scratch(dev, stream, kScratchBatch, host.size(), &scratch);
+        if (st != ENEC_OK) return st;
+        // pageable source: the call returns once the bytes are staged, so `host` may go out of scope
+        if (cudaMemcpyAsync(scratch, host.data(), host.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return ENEC_ERR_CUDA;
+        batch.jobs = reinterpret_cast<const DecodeJob*>(scratch);
+        batch.prefix = reinterpret_cast<const uint32_t*>(scratch + jobs_bytes);
+    }
     return dt == ENEC_BF16 ? launch_decode<ENEC_BF16>(batch, d_status, stream)
                            : launch_decode<ENEC_FP16>(batch, d_status, stream);
 }

@@ -568,19 +568,22 @@ struct BlockDesc {
 };
 static_assert(sizeof(BlockDesc) <= kStageMetaBytes, "descriptor fits the stage's meta area");
 
+constexpr uint32_t kInlineJobs = 16;  // tensors of a short batch that fit the kernel's parameter space
+
 // A launch decodes the blocks of one tensor or of a list of tensors. Blocks of all tensors form one
 // index space; a CTA takes a contiguous range of it, so it changes tensor rarely.
 struct DecodeBatch {
-    const DecodeJob* jobs;    // device array, or null for a single tensor
-    const uint32_t* prefix;   // device array [n_jobs + 1]: blocks before each tensor
+    const DecodeJob* jobs;    // device array, or null when the tensors travel inside the launch parameters
+    const uint32_t* prefix;   // device array [n_jobs + 1]: blocks before each tensor (null with jobs)
     uint32_t n_jobs;
     uint32_t total_blocks;
-    DecodeJob single;         // the tensor when jobs is null
+    DecodeJob inline_jobs[kInlineJobs];          // used when jobs is null (one tensor, or a short list)
+    uint32_t inline_prefix[kInlineJobs + 1];
 };
 
 template <int DT>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
-enec_decode_kernel(DecodeBatch batch, int* status) {
+enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     extern __shared__ __align__(128) uint8_t smem[];
     DecodeShared* ctl = reinterpret_cast<DecodeShared*>(smem);
     const uint32_t stages = smem_u32(smem) + uint32_t(sizeof(DecodeShared));
@@ -589,9 +592,9 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
     pdl_launch_dependents();
     pdl_wait();  // nothing above touches global memory
     if (batch.total_blocks == 0) {  // nothing to decode: only check the header of a single empty tensor
-        if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr) {
+        if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr && batch.n_jobs == 1) {
             JobCtx jc;
-            const int err = load_job<DT>(batch.single, jc);
+            const int err = load_job<DT>(batch.inline_jobs[0], jc);
             if (err) report(status, err);
         }
         return;
@@ -618,16 +621,18 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
         if (lane != 0) return;
         // the tensor that holds first_block
         uint32_t j = 0;
-        if (batch.jobs) {
+        const DecodeJob* jobs = batch.jobs ? batch.jobs : batch.inline_jobs;
+        const uint32_t* prefix = batch.jobs ? batch.prefix : batch.inline_prefix;
+        {
             uint32_t lo = 0, hi = batch.n_jobs;  // largest j with prefix[j] <= first_block
             while (hi - lo > 1) {
                 const uint32_t mid = (lo + hi) >> 1;
-                if (batch.prefix[mid] <= first_block) lo = mid; else hi = mid;
+                if (prefix[mid] <= first_block) lo = mid; else hi = mid;
             }
             j = lo;
         }
-        uint32_t job_first = batch.jobs ? batch.prefix[j] : 0;
-        uint32_t job_end = batch.jobs ? batch.prefix[j + 1] : batch.total_blocks;
+        uint32_t job_first = prefix[j];
+        uint32_t job_end = prefix[j + 1];
         bool parsed = false;
         JobCtx jc;
         StageLayout L;
@@ -641,13 +646,13 @@ enec_decode_kernel(DecodeBatch batch, int* status) {
             while (gb >= job_end) {  // next tensor (tensors without blocks are skipped)
                 ++j;
                 job_first = job_end;
-                job_end = batch.prefix[j + 1];
+                job_end = prefix[j + 1];
                 parsed = false;
             }
             const uint32_t k = gb - job_first;
             uint32_t t0;
             if (!parsed) {
-                const DecodeJob job = batch.jobs ? batch.jobs[j] : batch.single;
+                const DecodeJob job = jobs[j];
                 // the table sits right behind the header: fetch the block's two entries along with the
                 // header instead of after it (they are only used once the header has been checked)
                 uint32_t e0 = 0, e1 = 0;
