@@ -66,63 +66,35 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p) {
 // ---------------------------------------------------------------------------------------------------
 // Sec. 5.5 phase 1: histogram of the exponent field.
 //
-// Each lane keeps private 8-bit counters in shared memory (four bins per 32-bit word, the word's bank
-// equal to the lane), so counting needs neither atomics nor bank conflicts whatever the distribution;
-// a warp folds its counters into the CTA's 32-bit histogram every 28 loads of eight values (224 < 256).
+// Every warp keeps eight copies of the histogram in shared memory (lane l adds to copy l mod 8; a bin's
+// eight 32-bit counters fill one 32-byte row), so the adds of a warp instruction spread over all banks and
+// at most four lanes can meet on a counter. Counting is one `red.shared.add` per value: no read-modify-
+// write chain in the thread, no overflow, nothing to fold until the end.
 // ---------------------------------------------------------------------------------------------------
 template <int DT>
 struct HistShape {
     static constexpr int E = DT == ENEC_BF16 ? 8 : 5;
     static constexpr int kBins = 1 << E;
-    static constexpr int kQuads = kBins / 4;             // words per lane
-    static constexpr int kWarpBytes = kQuads * 128;      // counters of one warp
+    static constexpr int kCopies = 8;                    // copies of the histogram per warp
+    static constexpr int kWarpBytes = kBins * kCopies * 4;
 };
 
-// byte address (inside the warp's area) of lane `lane4 / 4`'s counter for exponent x
-template <int DT>
-__device__ __forceinline__ uint32_t counter_offset(uint32_t x) {
-    constexpr int Q = HistShape<DT>::kQuads;
-    return ((x & (Q - 1)) << 7) + (x / Q);
+// One value counted: a fire-and-forget shared-memory add on the copy of the warp's histogram that the lane
+// uses (eight copies per warp, 32 bytes per bin), addressed straight from the word's bits.
+__device__ __forceinline__ void red_add_one(uint32_t addr) {
+    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(addr), "r"(1u) : "memory");
 }
 
 template <int DT>
 __device__ __forceinline__ void count_word_pair(uint32_t base, uint32_t w) {
-    // two 16-bit values per 32-bit word; the counter's offset is taken straight from the word's bits
-    uint32_t a0, a1;
+    // two 16-bit values per 32-bit word; bin x sits at byte x * 32 of the warp's area
     if (DT == ENEC_BF16) {
-        // exponent x = bits 14..7: offset = (x & 63) << 7 | x >> 6 = (w & 0x1F80) + (bits 14..13)
-        a0 = base + (w & 0x1F80u) + ((w >> 13) & 3u);
-        a1 = base + ((w >> 16) & 0x1F80u) + ((w >> 29) & 3u);
+        red_add_one(base + ((w >> 2) & 0x1FE0u));    // x = bits 14..7
+        red_add_one(base + ((w >> 18) & 0x1FE0u));
     } else {
-        // exponent x = bits 14..10: offset = (x & 7) << 7 | x >> 3
-        a0 = base + ((w >> 3) & 0x380u) + ((w >> 13) & 3u);
-        a1 = base + ((w >> 19) & 0x380u) + ((w >> 29) & 3u);
+        red_add_one(base + ((w >> 5) & 0x3E0u));     // x = bits 14..10
+        red_add_one(base + ((w >> 21) & 0x3E0u));
     }
-    sts8(a0, lds8(a0) + 1);
-    sts8(a1, lds8(a1) + 1);
-}
-
-template <int DT>
-__device__ __forceinline__ void flush_counters(uint32_t warp_base, uint32_t lane, uint32_t* cta_hist) {
-    constexpr int Q = HistShape<DT>::kQuads;
-    __syncwarp();
-    for (uint32_t qd = lane; qd < uint32_t(Q); qd += 32) {
-        uint32_t even = 0, odd = 0;  // 16-bit sums of counter bytes 0|2 and 1|3
-#pragma unroll 8
-        for (uint32_t r = 0; r < 32; ++r) {
-            const uint32_t a = warp_base + qd * 128 + ((r + lane) & 31) * 4;
-            const uint32_t v = lds32(a);
-            even += v & 0x00FF00FFu;
-            odd += (v >> 8) & 0x00FF00FFu;
-            sts32(a, 0);
-        }
-        // counter byte s of quad qd belongs to bin s * Q + qd
-        if (even & 0xFFFFu) atomicAdd(&cta_hist[0 * Q + qd], even & 0xFFFFu);
-        if (odd & 0xFFFFu) atomicAdd(&cta_hist[1 * Q + qd], odd & 0xFFFFu);
-        if (even >> 16) atomicAdd(&cta_hist[2 * Q + qd], even >> 16);
-        if (odd >> 16) atomicAdd(&cta_hist[3 * Q + qd], odd >> 16);
-    }
-    __syncwarp();
 }
 
 __host__ __device__ inline int bit_width_u32(uint32_t v) {
@@ -224,7 +196,7 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     pdl_wait();  // nothing above touches global memory
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t warp_base = smem_u32(smem) + warp * kWarpBytes;
-    const uint32_t base = warp_base + lane * 4;
+    const uint32_t base = warp_base + (lane & 7) * 4;
     for (uint32_t i = tid; i < uint32_t(kWarpBytes / 4) * (kHistThreads / 32); i += kHistThreads)
         reinterpret_cast<uint32_t*>(smem)[i] = 0;
     cta_hist[tid] = 0;
@@ -235,7 +207,6 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     // a warp takes 2 KB at a time: four 16-byte loads per lane in flight before any counting
     constexpr uint32_t kUnroll = 4;
     const uint64_t warps_total = uint64_t(gridDim.x) * (kHistThreads / 32);
-    uint32_t since_flush = 0;
     for (uint64_t first = (uint64_t(blockIdx.x) * (kHistThreads / 32) + warp) * (32 * kUnroll); first < nchunks;
          first += warps_total * (32 * kUnroll)) {
         uint4 v[kUnroll];
@@ -256,12 +227,18 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
                 count_word_pair<DT>(base, v[u].w);
             }
         }
-        if (++since_flush == 7) {  // 7 * 4 * 8 = 224 values per lane since the last flush, below 256
-            flush_counters<DT>(warp_base, lane, cta_hist);
-            since_flush = 0;
-        }
     }
-    flush_counters<DT>(warp_base, lane, cta_hist);
+    __syncthreads();
+    if (tid < uint32_t(HistShape<DT>::kBins)) {  // fold the warps' copies of bin `tid`
+        uint32_t sum = 0;
+        for (uint32_t wp = 0; wp < kHistThreads / 32; ++wp) {
+            const uint32_t row = smem_u32(smem) + wp * kWarpBytes + tid * 32;
+            const uint4 lo = lds128(row), hi = lds128(row + 16);
+            sum += lo.x + lo.y + lo.z + lo.w + hi.x + hi.y + hi.z + hi.w;
+        }
+        cta_hist[tid] = sum;
+    }
+    __syncthreads();
     if (blockIdx.x == 0 && tid == 0) {  // the last count mod 8 values
         constexpr int sh = DT == ENEC_BF16 ? 7 : 10;
         for (uint64_t e = nchunks << 3; e < count; ++e)
