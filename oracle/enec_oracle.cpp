@@ -6,7 +6,8 @@
  *
  * Stream layout (this repository's definition; little-endian; every section starts on a 16-byte
  * boundary and is zero padded):
- *   header 64 B | table u32[nblocks+1] | mask | low plane | (fp16: sm-hi plane) | sm plane | high records
+ *   header 64 B | table u32[nblocks+1] | mask | low plane | (fp16: sm-hi plane) | sm plane |
+ *   (fp32: sm-lo plane, mantissa bits 15..0, two bytes per element) | high records
  */
 #include "enec_oracle.h"
 
@@ -22,7 +23,9 @@ constexpr size_t kHeaderBytes = 64;
 enum { OK = 0, ERR_INVALID_ARG = -1, ERR_UNSUPPORTED_DTYPE = -2, ERR_BUFFER_TOO_SMALL = -3,
        ERR_BAD_STREAM = -4, ERR_PARAMS_NOT_LOSSLESS = -5 };
 
-int exp_bits(int dtype) { return dtype == 0 ? 8 : 5; }
+int exp_bits(int dtype) { return dtype == 1 ? 5 : 8; }  // bf16 and fp32: 8 exponent bits; fp16: 5
+
+bool known_dtype(int dtype) { return dtype >= 0 && dtype <= 2; }
 
 size_t align16(size_t v) { return (v + 15) & ~size_t(15); }
 
@@ -69,7 +72,7 @@ Geometry geometry(size_t count) {
 }
 
 struct Sections {
-    size_t table, mask, low, smhi, sm, high, total;
+    size_t table, mask, low, smhi, sm, smlo, high, total;
 };
 
 // Section offsets for stored widths (n, m) and a_total anomalous groups.
@@ -80,7 +83,8 @@ Sections sections(int dtype, size_t count, const Geometry& g, int n, int m, uint
     s.low = s.mask + align16((size_t(g.total_groups) + 7) / 8);
     s.smhi = s.low + align16(size_t(g.padded_count) * m / 8);
     s.sm = s.smhi + (dtype == 1 ? align16(size_t(g.padded_count) * 3 / 8) : 0);
-    s.high = s.sm + align16(count);
+    s.smlo = s.sm + align16(count);
+    s.high = s.smlo + (dtype == 2 ? align16(count * 2) : 0);
     s.total = s.high + align16(size_t(a_total) * 2 * (n - m));
     return s;
 }
@@ -255,31 +259,40 @@ bool params_lossless(int b, int n, int l, int h, int E) {
     return true;
 }
 
-void split(uint16_t w, int dtype, uint32_t* x, uint32_t* sm) {
-    if (dtype == 0) { *x = (w >> 7) & 0xFF; *sm = ((w >> 8) & 0x80) | (w & 0x7F); }
+// Sec. 4.2 "Split". fp32 keeps its 24 sign/mantissa bits as they are, as the text says of all formats; the
+// exponent goes the same way as bf16's (Sec. 6.2: "we avoid compressing the mantissa").
+void split(uint32_t w, int dtype, uint32_t* x, uint32_t* sm) {
+    if (dtype == 2) { *x = (w >> 23) & 0xFF; *sm = ((w >> 8) & 0x800000) | (w & 0x7FFFFF); }
+    else if (dtype == 0) { *x = (w >> 7) & 0xFF; *sm = ((w >> 8) & 0x80) | (w & 0x7F); }
     else            { *x = (w >> 10) & 0x1F; *sm = ((w >> 5) & 0x400) | (w & 0x3FF); }
 }
 
-uint16_t join(uint32_t x, uint32_t sm, int dtype) {
-    if (dtype == 0) return uint16_t(((sm & 0x80) << 8) | (x << 7) | (sm & 0x7F));
-    return uint16_t(((sm & 0x400) << 5) | (x << 10) | (sm & 0x3FF));
+uint32_t join(uint32_t x, uint32_t sm, int dtype) {
+    if (dtype == 2) return ((sm & 0x800000) << 8) | (x << 23) | (sm & 0x7FFFFF);
+    if (dtype == 0) return ((sm & 0x80) << 8) | (x << 7) | (sm & 0x7F);
+    return ((sm & 0x400) << 5) | (x << 10) | (sm & 0x3FF);
 }
 
-int encode(const uint16_t* in, int dtype, size_t count, bool have_params, int b, int n, int m,
+// Element i of a tensor of 16-bit (bf16, fp16) or 32-bit (fp32) words.
+uint32_t load_word(const void* in, int dtype, size_t i) {
+    return dtype == 2 ? static_cast<const uint32_t*>(in)[i] : static_cast<const uint16_t*>(in)[i];
+}
+
+int encode(const void* in, int dtype, size_t count, bool have_params, int b, int n, int m,
            uint8_t* out, size_t capacity, size_t* out_size) {
-    if (dtype != 0 && dtype != 1) return ERR_UNSUPPORTED_DTYPE;
+    if (!known_dtype(dtype)) return ERR_UNSUPPORTED_DTYPE;
     if ((!in && count) || !out || !out_size || (count >> 36)) return ERR_INVALID_ARG;
     const int E = exp_bits(dtype);
     const Geometry g = geometry(count);
 
     // step 1: split; phase 1: histogram of the exponent field
     std::vector<uint8_t> x(count);
-    std::vector<uint16_t> sm(count);
+    std::vector<uint32_t> sm(count);
     std::vector<uint64_t> hist(size_t(1) << E, 0);
     for (size_t i = 0; i < count; ++i) {
         uint32_t xe, s;
-        split(in[i], dtype, &xe, &s);
-        x[i] = uint8_t(xe); sm[i] = uint16_t(s);
+        split(load_word(in, dtype, i), dtype, &xe, &s);
+        x[i] = uint8_t(xe); sm[i] = s;
         hist[xe] += 1;
     }
     if (!have_params) {
@@ -349,13 +362,21 @@ int encode(const uint16_t* in, int dtype, size_t count, bool have_params, int b,
     if (!mask.empty()) std::memcpy(out + s.mask, mask.data(), mask.size());
     if (!low.empty()) std::memcpy(out + s.low, low.data(), low.size());
     if (!smhi.empty()) std::memcpy(out + s.smhi, smhi.data(), smhi.size());
-    for (size_t i = 0; i < count; ++i) out[s.sm + i] = uint8_t(sm[i] & 0xFF);
+    if (dtype == 2) {
+        // fp32: sign | mantissa bits 22..16 in the byte plane, mantissa bits 15..0 in the two-byte plane
+        for (size_t i = 0; i < count; ++i) {
+            out[s.sm + i] = uint8_t(sm[i] >> 16);
+            put_u16(out + s.smlo + 2 * i, uint16_t(sm[i] & 0xFFFF));
+        }
+    } else {
+        for (size_t i = 0; i < count; ++i) out[s.sm + i] = uint8_t(sm[i] & 0xFF);
+    }
     if (!high.empty()) std::memcpy(out + s.high, high.data(), high.size());
     return OK;
 }
 
-int decode(const uint8_t* in, size_t in_size, int dtype, size_t count, uint16_t* out) {
-    if (dtype != 0 && dtype != 1) return ERR_UNSUPPORTED_DTYPE;
+int decode(const uint8_t* in, size_t in_size, int dtype, size_t count, void* out) {
+    if (!known_dtype(dtype)) return ERR_UNSUPPORTED_DTYPE;
     if (!in || (!out && count)) return ERR_INVALID_ARG;
     if (in_size < kHeaderBytes + 16) return ERR_BAD_STREAM;
     if (std::memcmp(in, "ENEC", 4) != 0 || get_u16(in + 4) != 1) return ERR_BAD_STREAM;
@@ -396,7 +417,12 @@ int decode(const uint8_t* in, size_t in_size, int dtype, size_t count, uint16_t*
             uint32_t xe = inverse_transform(y[i], b, n, E);
             uint32_t smv = in[s.sm + first + i];
             if (dtype == 1) smv |= uint32_t(hi3[i]) << 8;
-            out[first + i] = join(xe, smv, dtype);
+            if (dtype == 2) {
+                smv = (smv << 16) | get_u16(in + s.smlo + 2 * (first + i));
+                static_cast<uint32_t*>(out)[first + i] = join(xe, smv, dtype);
+            } else {
+                static_cast<uint16_t*>(out)[first + i] = uint16_t(join(xe, smv, dtype));
+            }
         }
     }
     return OK;
@@ -406,8 +432,8 @@ int decode(const uint8_t* in, size_t in_size, int dtype, size_t count, uint16_t*
 
 extern "C" {
 
-void enec_oracle_split(uint16_t w, int dtype, uint32_t* x, uint32_t* sm) { split(w, dtype, x, sm); }
-uint16_t enec_oracle_join(uint32_t x, uint32_t sm, int dtype) { return join(x, sm, dtype); }
+void enec_oracle_split(uint32_t w, int dtype, uint32_t* x, uint32_t* sm) { split(w, dtype, x, sm); }
+uint32_t enec_oracle_join(uint32_t x, uint32_t sm, int dtype) { return join(x, sm, dtype); }
 int enec_oracle_width_eq1(int b, int l, int h, int E) { return width_eq1(b, l, h, E); }
 uint32_t enec_oracle_transform(uint32_t x, int b, int n) { return transform(x, b, n); }
 uint32_t enec_oracle_inverse_transform(uint32_t y, int b, int n, int E) { return inverse_transform(y, b, n, E); }
@@ -429,7 +455,7 @@ void enec_oracle_alg2_unpack(const uint8_t* in, size_t N, int a, uint16_t* out) 
 }
 
 size_t enec_oracle_max_compressed_size(int dtype, size_t count) {
-    if ((dtype != 0 && dtype != 1) || (count >> 36)) return 0;
+    if (!known_dtype(dtype) || (count >> 36)) return 0;
     const int E = exp_bits(dtype);
     const Geometry g = geometry(count);
     size_t worst = 0;  // widest stored width, every group anomalous, every split m
@@ -441,18 +467,18 @@ size_t enec_oracle_max_compressed_size(int dtype, size_t count) {
 }
 
 int enec_oracle_compress(const void* in, int dtype, size_t count, void* out, size_t capacity, size_t* out_size) {
-    return encode(static_cast<const uint16_t*>(in), dtype, count, false, 0, 0, 0,
+    return encode(in, dtype, count, false, 0, 0, 0,
                   static_cast<uint8_t*>(out), capacity, out_size);
 }
 
 int enec_oracle_compress_with_params(const void* in, int dtype, size_t count, int b, int n, int m, void* out,
                                      size_t capacity, size_t* out_size) {
-    return encode(static_cast<const uint16_t*>(in), dtype, count, true, b, n, m,
+    return encode(in, dtype, count, true, b, n, m,
                   static_cast<uint8_t*>(out), capacity, out_size);
 }
 
 int enec_oracle_decompress(const void* in, size_t in_size, int dtype, size_t count, void* out) {
-    return decode(static_cast<const uint8_t*>(in), in_size, dtype, count, static_cast<uint16_t*>(out));
+    return decode(static_cast<const uint8_t*>(in), in_size, dtype, count, out);
 }
 
 }  // extern "C"

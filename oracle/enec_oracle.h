@@ -21,11 +21,11 @@
 extern "C" {
 #endif
 
-/* dtype: 0 = bf16, 1 = fp16. Status: 0 ok, negative = error (same numbering as the CUDA library). */
+/* dtype: 0 = bf16, 1 = fp16, 2 = fp32 (32-bit words). Status: 0 ok, negative = error (same numbering as the CUDA library). */
 
-/* Sec. 4.2 "Split": exponent field and sign/mantissa remainder of one 16-bit word. */
-void enec_oracle_split(uint16_t w, int dtype, uint32_t* x, uint32_t* sm);
-uint16_t enec_oracle_join(uint32_t x, uint32_t sm, int dtype);
+/* Sec. 4.2 "Split": exponent field and sign/mantissa remainder of one word (16 bits, or 32 for fp32). */
+void enec_oracle_split(uint32_t w, int dtype, uint32_t* x, uint32_t* sm);
+uint32_t enec_oracle_join(uint32_t x, uint32_t sm, int dtype);
 
 /* Eq. 1: stored width n (sign bit included) for mapping parameter b and occupied range [l, h]. */
 int enec_oracle_width_eq1(int b, int l, int h, int E);

@@ -12,7 +12,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
-BF16, FP16 = 0, 1
+BF16, FP16, FP32 = 0, 1, 2
 
 
 def lib():
@@ -23,10 +23,10 @@ def lib():
         mod = importlib.util.module_from_spec(spec)
         spec.loader.exec_module(mod)
         L = C.CDLL(mod.build())
-        L.enec_oracle_split.argtypes = [C.c_uint16, C.c_int, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+        L.enec_oracle_split.argtypes = [C.c_uint32, C.c_int, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
         L.enec_oracle_split.restype = None
         L.enec_oracle_join.argtypes = [C.c_uint32, C.c_uint32, C.c_int]
-        L.enec_oracle_join.restype = C.c_uint16
+        L.enec_oracle_join.restype = C.c_uint32
         L.enec_oracle_width_eq1.argtypes = [C.c_int] * 4
         L.enec_oracle_width_eq1.restype = C.c_int
         L.enec_oracle_transform.argtypes = [C.c_uint32, C.c_int, C.c_int]
@@ -113,8 +113,9 @@ def max_compressed_size(dtype, count):
 
 
 def compress(words, dtype, params=None):
-    """words: numpy uint16 array (raw bf16/fp16 bit patterns). Returns the stream as a uint8 array."""
-    words = np.ascontiguousarray(words, dtype=np.uint16).reshape(-1)
+    """words: numpy array of raw bit patterns (uint16 for bf16/fp16, uint32 for fp32). Returns the stream as a
+    uint8 array."""
+    words = np.ascontiguousarray(words, dtype=np.uint32 if dtype == FP32 else np.uint16).reshape(-1)
     cap = max_compressed_size(dtype, words.size)
     out = np.empty(cap, dtype=np.uint8)
     size = C.c_size_t(0)
@@ -131,7 +132,7 @@ def compress(words, dtype, params=None):
 
 def decompress(stream, dtype, count):
     stream = np.ascontiguousarray(stream, dtype=np.uint8)
-    out = np.empty(count, dtype=np.uint16)
+    out = np.empty(count, dtype=np.uint32 if dtype == FP32 else np.uint16)
     st = lib().enec_oracle_decompress(stream.ctypes.data, stream.size, dtype, count, out.ctypes.data)
     if st != 0:
         raise OracleError(st)

@@ -403,3 +403,73 @@ def test_decoder_rejects_damaged_streams(oracle):
         oracle.decompress(s[:-16], 0, words.size)
     with pytest.raises(oracle.OracleError):
         oracle.decompress(s, 1, words.size)
+
+
+# ---------------------------------------------------------------- fp32 (Sec. 6.2: the mantissa is not compressed)
+def test_fp32_split_fields(oracle):
+    # 1.0f = 0x3F800000: exponent 127; -2.5f = 0xC0200000: sign 1, exponent 128, mantissa 0x200000
+    assert oracle.split(0x3F800000, 2) == (127, 0)
+    assert oracle.split(0xC0200000, 2) == (128, 0x800000 | 0x200000)
+    rng = np.random.default_rng(31)
+    for w in rng.integers(0, 1 << 32, 4000, dtype=np.uint64):
+        x, sm = oracle.split(int(w), 2)
+        assert oracle.join(x, sm, 2) == int(w)
+    vals = rng.normal(0, 0.02, 300).astype(np.float32)
+    for v, w in zip(vals, vals.view(np.uint32)):
+        _, e = np.frexp(np.float64(v))
+        assert oracle.split(int(w), 2)[0] == e - 1 + 127          # exponent field = floor(log2 |v|) + bias
+
+
+def test_fp32_stream_hand(oracle):
+    fx = read_fixture("stream_hand_fp32.txt")
+    words = np.array([int(t, 16) for t in fx["words"][0].split()], dtype=np.uint32)
+    expect = np.concatenate([hexbytes(fx[k][0]) for k in ("header", "table", "mask", "low", "sm", "smlo")])
+    got = oracle.compress(words, 2)
+    assert got.tolist() == expect.tolist()
+    assert oracle.decompress(got, 2, 16).tolist() == words.tolist()
+
+
+def test_fp32_is_the_bf16_stream_of_the_high_halves_plus_raw_low_halves(oracle):
+    # an fp32 word's high half has bf16's layout, so the fp32 stream must be the bf16 stream of the high halves
+    # (same parameters, table, mask, planes, records) with the low halves stored as they are in between
+    rng = np.random.default_rng(32)
+    count = 3 * 16384 + 777
+    w = rng.normal(0, 0.02, count).astype(np.float32).view(np.uint32)
+    s32 = oracle.compress(w, 2)
+    s16 = oracle.compress((w >> 16).astype(np.uint16), 0)
+    a16 = lambda v: (v + 15) // 16 * 16
+    high_bytes = int(s16[32:36].view(np.uint32)[0]) * 2 * (int(s16[21]) - int(s16[22]))
+    cut = s16.size - a16(high_bytes)                          # where the bf16 stream's records start
+    assert s32[20:24].tolist() == s16[20:24].tolist()          # b, n, m, L
+    assert s32[64:cut].tolist() == s16[64:cut].tolist()        # table, mask, low plane, byte plane
+    lo = s32[cut:cut + 2 * count].view(np.uint16)
+    assert lo.tolist() == (w & 0xFFFF).astype(np.uint16).tolist()
+    assert s32[cut + a16(2 * count):].tolist() == s16[cut:].tolist()   # records
+    assert s32.size == s16.size + a16(2 * count)
+    assert int(s32[40:48].view(np.uint64)[0]) == s32.size and s32[6] == 2
+
+
+def test_fp32_special_values_and_tails_roundtrip(oracle):
+    rng = np.random.default_rng(33)
+    special = np.array([0x00000000, 0x80000000, 0x7F800000, 0xFF800000, 0x7FC00001, 0x00000001, 0x007FFFFF,
+                        0x7F7FFFFF, 0xFFFFFFFF, 0x3F800000], dtype=np.uint32)
+    for count in (0, 1, 15, 16, 17, 1000, 16384, 16385, 2 * 16384 + 4097):
+        w = rng.integers(0, 1 << 32, count, dtype=np.uint64).astype(np.uint32)
+        w[: min(count, special.size)] = special[: min(count, special.size)]
+        s = oracle.compress(w, 2)
+        assert s.size % 16 == 0 and s.size <= oracle.max_compressed_size(2, count)
+        assert np.array_equal(oracle.decompress(s, 2, count), w)
+    with pytest.raises(oracle.OracleError):
+        oracle.decompress(oracle.compress(special, 2), 0, special.size)
+
+
+def test_fp32_gaussian_lands_on_table5_and_table4(oracle):
+    # Table 5: fp32 models use (121..125, 6, 3, 16); Table 4: ratio 1.15 for the fp32 models
+    fx = read_fixture("table5_params.txt")
+    rows = [tuple(map(int, fx[k][0].split())) for k in ("OLMo", "BERT", "Wav2Vec")]
+    assert {r[1:] for r in rows} == {(6, 3, 16)}
+    rng = np.random.default_rng(34)
+    w = rng.normal(0, 0.02, 1 << 21).astype(np.float32).view(np.uint32)
+    s = oracle.compress(w, 2)
+    assert 119 <= int(s[20]) <= 125 and (int(s[21]), int(s[22])) == (6, 3)
+    assert 1.13 < w.nbytes / s.size < 1.18
