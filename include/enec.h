@@ -1,5 +1,5 @@
 /*
- * libenec -- ENEC lossless codec for bf16/fp16 model weights on NVIDIA B200 (sm_100a).
+ * libenec -- ENEC lossless codec for bf16/fp16 (and fp32) model weights on NVIDIA B200 (sm_100a).
  *
  * Block-based fixed-length coding: every 16-bit value is split into its exponent field and its
  * sign/mantissa bits (Sec. 4.2, Algorithm 1 "Split"); exponents go through the branch-free integer
@@ -7,7 +7,9 @@
  * with m bits per element, or with n bits when its OR needs more than m (Sec. 5.2); bits are packed with
  * hierarchical halving bit-packing (Algorithm 2); a prefix sum over the per-block counts of wide groups
  * gives every block's offset in the variable-length part of the stream (Sec. 5.1, Sec. 5.4); (b, n, m) are
- * chosen per tensor from the exponent histogram (Sec. 5.5, Eq. 1, 3, 4).
+ * chosen per tensor from the exponent histogram (Sec. 5.5, Eq. 1, 3, 4). fp32 values (32-bit words) take the same
+ * path as bf16 with their high halves; their low halves are stored as they are (Sec. 6.2: the mantissa is not
+ * compressed). `count` is always a number of elements.
  *
  * All pointers named d_* are DEVICE pointers, 16-byte aligned, owned by the caller. Every call only
  * enqueues work on `stream` and returns; nothing synchronises with the host. Errors the host can see
@@ -30,7 +32,7 @@
 extern "C" {
 #endif
 
-typedef enum { ENEC_BF16 = 0, ENEC_FP16 = 1 } enec_dtype;
+typedef enum { ENEC_BF16 = 0, ENEC_FP16 = 1, ENEC_FP32 = 2 } enec_dtype;
 
 typedef enum {
     ENEC_OK = 0,

@@ -8,8 +8,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libenec.so")
 _LIB = None
 
-BF16, FP16 = 0, 1
-_DT = {torch.bfloat16: BF16, torch.float16: FP16}
+BF16, FP16, FP32 = 0, 1, 2
+_DT = {torch.bfloat16: BF16, torch.float16: FP16, torch.float32: FP32}
 
 STATUS_NAMES = {0: "ENEC_OK", -1: "ENEC_ERR_INVALID_ARG", -2: "ENEC_ERR_UNSUPPORTED_DTYPE",
                 -3: "ENEC_ERR_BUFFER_TOO_SMALL", -4: "ENEC_ERR_BAD_STREAM",
@@ -106,7 +106,7 @@ def enec_launch_count() -> int:
 
 # ---- convenience wrappers (allocation with torch, status check) --------------------------------------
 def compress_tensor(t: torch.Tensor, params=None) -> torch.Tensor:
-    """Compresses a CUDA bf16/fp16 tensor; returns the stream as a uint8 CUDA tensor (synchronises once to
+    """Compresses a CUDA bf16/fp16/fp32 tensor; returns the stream as a uint8 CUDA tensor (synchronises once to
     read the stream length)."""
     dt = _DT[t.dtype]
     t = t.contiguous()

@@ -14,9 +14,9 @@ std::atomic<uint64_t> g_launches{0};
 
 struct DeviceInfo {
     int sms = 0;
-    bool decode_attr_set[2] = {false, false};
-    bool hist_attr_set[2] = {false, false};
-    bool encode_attr_set[2] = {false, false};
+    bool decode_attr_set[3] = {false, false, false};
+    bool hist_attr_set[3] = {false, false, false};
+    bool encode_attr_set[3] = {false, false, false};
 };
 
 static DeviceInfo& device_info(int dev) {
@@ -105,7 +105,7 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
                 return ENEC_ERR_CUDA;
             info.hist_attr_set[DT] = true;
         }
-        const uint64_t chunks = job.count >> 3;
+        const uint64_t chunks = (job.count * uint64_t(elem_bytes(DT))) >> 4;  // 16-byte loads
         uint64_t grid = (chunks + kHistThreads - 1) / kHistThreads;
         if (grid > uint64_t(info.sms) * 3) grid = uint64_t(info.sms) * 3;
         if (grid == 0) grid = 1;
@@ -130,7 +130,7 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
 static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count, bool with_params, int b, int n,
                                    int m, void* d_out, size_t out_capacity, size_t* d_out_size, int* d_status,
                                    cudaStream_t stream) {
-    if (dt != ENEC_BF16 && dt != ENEC_FP16) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if ((!d_in && count) || !d_out || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out) ||
         (reinterpret_cast<uintptr_t>(d_out_size) & 7))
         return ENEC_ERR_INVALID_ARG;
@@ -164,8 +164,9 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
     job.b = b; job.n = n; job.m = m;
     job.from_search = with_params ? 0 : 1;
     job.check = with_params ? 1 : 0;
-    return dt == ENEC_BF16 ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream)
-                           : launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream);
+    return dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream)
+           : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream)
+                             : launch_encode<ENEC_FP32>(job, g.nblocks, !with_params, d_status, info, stream);
 }
 
 // ---- compression without any allocation ------------------------------------------------------------
@@ -199,7 +200,7 @@ using namespace enec;
 extern "C" {
 
 size_t enec_max_compressed_size(enec_dtype dt, size_t count) {
-    if ((dt != ENEC_BF16 && dt != ENEC_FP16) || (uint64_t(count) >> 36)) return 0;
+    if (!known_dtype(dt) || (uint64_t(count) >> 36)) return 0;
     const int E = exp_bits(dt);
     const Geometry g = make_geometry(count);
     uint64_t worst = 0;
@@ -212,7 +213,7 @@ size_t enec_max_compressed_size(enec_dtype dt, size_t count) {
 
 enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
                             int* d_status, enec_stream_t stream) {
-    if (dt != ENEC_BF16 && dt != ENEC_FP16) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if (!d_in || (!d_out && count) || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out))
         return ENEC_ERR_INVALID_ARG;
     if (in_size < kHeaderBytes + 16) return ENEC_ERR_BAD_STREAM;
@@ -225,13 +226,14 @@ enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, siz
                                      uint64_t(in_size)};
     batch.inline_prefix[0] = 0;
     batch.inline_prefix[1] = batch.total_blocks;
-    return dt == ENEC_BF16 ? launch_decode<ENEC_BF16>(batch, d_status, stream)
-                           : launch_decode<ENEC_FP16>(batch, d_status, stream);
+    return dt == ENEC_BF16   ? launch_decode<ENEC_BF16>(batch, d_status, stream)
+           : dt == ENEC_FP16 ? launch_decode<ENEC_FP16>(batch, d_status, stream)
+                             : launch_decode<ENEC_FP32>(batch, d_status, stream);
 }
 
 enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, int* d_status,
                                     enec_stream_t stream) {
-    if (dt != ENEC_BF16 && dt != ENEC_FP16) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if (n_items < 0 || (n_items > 0 && !h_items)) return ENEC_ERR_INVALID_ARG;
     if (n_items == 0) return ENEC_OK;
     // descriptors and block prefix in one host buffer: [jobs | prefix]
@@ -276,8 +278,9 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
         batch.jobs = reinterpret_cast<const DecodeJob*>(scratch);
         batch.prefix = reinterpret_cast<const uint32_t*>(scratch + jobs_bytes);
     }
-    return dt == ENEC_BF16 ? launch_decode<ENEC_BF16>(batch, d_status, stream)
-                           : launch_decode<ENEC_FP16>(batch, d_status, stream);
+    return dt == ENEC_BF16   ? launch_decode<ENEC_BF16>(batch, d_status, stream)
+           : dt == ENEC_FP16 ? launch_decode<ENEC_FP16>(batch, d_status, stream)
+                             : launch_decode<ENEC_FP32>(batch, d_status, stream);
 }
 
 enec_status enec_compress(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
@@ -294,7 +297,7 @@ enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t co
 
 enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
                                   size_t* d_out_size, int* d_status, enec_stream_t stream) {
-    if (dt != ENEC_BF16 && dt != ENEC_FP16) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if (uint64_t(count) > kNoAllocMaxCount) return ENEC_ERR_TOO_LARGE;
     if ((!d_in && count) || !d_out || !aligned16(d_in) || !aligned16(d_out) ||
         (reinterpret_cast<uintptr_t>(d_out_size) & 7))
@@ -326,8 +329,9 @@ enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count,
     job.b = 0; job.n = 0; job.m = 0;
     job.from_search = 1;
     job.check = 0;
-    return dt == ENEC_BF16 ? launch_encode<ENEC_BF16>(job, g.nblocks, true, d_status, info, stream)
-                           : launch_encode<ENEC_FP16>(job, g.nblocks, true, d_status, info, stream);
+    return dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, true, d_status, info, stream)
+           : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, true, d_status, info, stream)
+                             : launch_encode<ENEC_FP32>(job, g.nblocks, true, d_status, info, stream);
 }
 
 uint64_t enec_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -34,7 +34,9 @@ struct alignas(16) Header {
 };
 static_assert(sizeof(Header) == 64, "header is 64 bytes");
 
-__host__ __device__ inline int exp_bits(int dt) { return dt == ENEC_BF16 ? 8 : 5; }
+__host__ __device__ constexpr bool known_dtype(int dt) { return dt == ENEC_BF16 || dt == ENEC_FP16 || dt == ENEC_FP32; }
+__host__ __device__ constexpr int exp_bits(int dt) { return dt == ENEC_FP16 ? 5 : 8; }
+__host__ __device__ constexpr int elem_bytes(int dt) { return dt == ENEC_FP32 ? 4 : 2; }
 __host__ __device__ inline uint64_t align16(uint64_t v) { return (v + 15) & ~uint64_t(15); }
 
 struct Geometry {
@@ -59,7 +61,7 @@ __host__ __device__ inline Geometry make_geometry(uint64_t count) {
 }
 
 struct Sections {
-    uint64_t table, mask, low, smhi, sm, high, total;
+    uint64_t table, mask, low, smhi, sm, smlo, high, total;
 };
 
 __host__ __device__ inline Sections make_sections(int dt, uint64_t count, const Geometry& g, int n, int m,
@@ -70,7 +72,8 @@ __host__ __device__ inline Sections make_sections(int dt, uint64_t count, const 
     s.low = s.mask + align16((uint64_t(g.total_groups) + 7) / 8);
     s.smhi = s.low + align16(g.padded_count * uint64_t(m) / 8);
     s.sm = s.smhi + (dt == ENEC_FP16 ? align16(g.padded_count * 3 / 8) : 0);
-    s.high = s.sm + align16(count);
+    s.smlo = s.sm + align16(count);  // fp32 only: mantissa bits 15..0, two bytes per element
+    s.high = s.smlo + (dt == ENEC_FP32 ? align16(count * 2) : 0);
     s.total = s.high + align16(a_total * 2 * uint64_t(n - m));
     return s;
 }
@@ -121,6 +124,11 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                      smem_u32(dst)),
                  "l"(src), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
+}
+// Asks for `bytes` of global memory to be brought into L2 (no destination, nothing to wait for).
+// src 16-byte aligned; bytes a positive multiple of 16.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {

@@ -177,7 +177,7 @@ struct JobCtx {
     uint32_t nblocks, tail_real, tail_padded;
     uint32_t a_total;
     int b, n, m;
-    uint64_t off_table, off_mask, off_low, off_smhi, off_sm, off_high, total;
+    uint64_t off_table, off_mask, off_low, off_smhi, off_sm, off_smlo, off_high, total;
 };
 
 // Reads and validates the header. Returns 0 or an enec_status.
@@ -188,7 +188,7 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
     if (h.magic != kMagic || h.version != kVersion || h.dtype != DT || h.count != job.count ||
         h.block != kBlockElems || h.L != kGroupElems)
         return ENEC_ERR_BAD_STREAM;
-    constexpr int E = DT == ENEC_BF16 ? 8 : 5;
+    constexpr int E = exp_bits(DT);
     if (h.n < 1 || h.n > E || h.m < 1 || h.m > h.n || h.b >= (1 << E)) return ENEC_ERR_BAD_STREAM;
     const Geometry g = make_geometry(job.count);
     if (h.nblocks != g.nblocks || h.total_groups != g.total_groups || h.a_total > g.total_groups)
@@ -203,7 +203,7 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
     c.a_total = h.a_total;
     c.b = h.b; c.n = h.n; c.m = h.m;
     c.off_table = s.table; c.off_mask = s.mask; c.off_low = s.low; c.off_smhi = s.smhi; c.off_sm = s.sm;
-    c.off_high = s.high; c.total = s.total;
+    c.off_smlo = s.smlo; c.off_high = s.high; c.total = s.total;
     return 0;
 }
 
@@ -240,7 +240,8 @@ struct RunCtx {
     uint32_t expanded;    // shared address: expanded records
     uint32_t cap;         // records expanded in shared memory
     const uint8_t* high;  // global: first record of the block
-    uint16_t* out;        // global: first element of the block
+    uint16_t* out;        // global: first element of the block (fp32: four bytes per element)
+    const uint16_t* lo;   // global, fp32 only: mantissa bits 15..0 of the block's elements
     uint32_t real;        // real elements in the block
     uint32_t c4_or_h, fix, s4, b4;  // packed transform constants
     uint32_t c4;                    // rep4(b + 2^(n-1)) when that sum fits a byte
@@ -272,6 +273,15 @@ __device__ __noinline__ uint2 record_half_from_global(const uint8_t* rp, uint32_
     return second_half ? make_uint2(v.z, v.w) : make_uint2(v.x, v.y);
 }
 
+// fp32: joins the high halves of eight values (w, element order) with their low halves and stores 32 bytes.
+__device__ __forceinline__ void store_fp32_run(uint32_t* out, uint4 w, uint4 lo) {
+    uint4* o = reinterpret_cast<uint4*>(out);
+    o[0] = make_uint4(prmt(lo.x, w.x, 0x5410u), prmt(lo.x, w.x, 0x7632u), prmt(lo.y, w.y, 0x5410u),
+                      prmt(lo.y, w.y, 0x7632u));
+    o[1] = make_uint4(prmt(lo.z, w.z, 0x5410u), prmt(lo.z, w.z, 0x7632u), prmt(lo.w, w.w, 0x5410u),
+                      prmt(lo.w, w.w, 0x7632u));
+}
+
 // Finishes eight consecutive elements e0 .. e0+7 of a block: high bits of wide groups, inverse transform,
 // rejoin with sign/mantissa, store.
 template <int DT, int M, int HB>
@@ -290,8 +300,8 @@ __device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, u
     const uint32_t x1 = inverse_transform4<DT>(r, y.y);
     const uint2 smv = lds64(r.sm + e0);
     uint32_t lo0, lo1, hi0, hi1;
-    if (DT == ENEC_BF16) {
-        // word = sign << 15 | x << 7 | mant7 ; sm byte = sign << 7 | mant7
+    if (DT != ENEC_FP16) {
+        // word = sign << 15 | x << 7 | mant7 ; sm byte = sign << 7 | mant7 (fp32: the high half of the value)
         hi0 = (smv.x & 0x80808080u) | ((x0 >> 1) & 0x7F7F7F7Fu);
         hi1 = (smv.y & 0x80808080u) | ((x1 >> 1) & 0x7F7F7F7Fu);
         lo0 = ((x0 << 7) & 0x80808080u) | (smv.x & 0x7F7F7F7Fu);
@@ -309,6 +319,18 @@ __device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, u
     w.z = prmt(lo1, hi1, 0x5140u);
     w.w = prmt(lo1, hi1, 0x7362u);
     if (!active) return;
+    if constexpr (DT == ENEC_FP32) {
+        uint32_t* out32 = reinterpret_cast<uint32_t*>(r.out) + e0;
+        if (e0 + 8 <= r.real) {
+            store_fp32_run(out32, w, __ldg(reinterpret_cast<const uint4*>(r.lo + e0)));
+        } else if (e0 < r.real) {
+            for (uint32_t i = 0; e0 + i < r.real; ++i) {
+                const uint32_t pair = (i >> 1) == 0 ? w.x : (i >> 1) == 1 ? w.y : (i >> 1) == 2 ? w.z : w.w;
+                out32[i] = ((pair >> (16 * (i & 1))) << 16) | r.lo[e0 + i];
+            }
+        }
+        return;
+    }
     if (e0 + 8 <= r.real) {
         *reinterpret_cast<uint4*>(r.out + e0) = w;
     } else if (e0 < r.real) {
@@ -367,6 +389,8 @@ __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_lo
     const uint32_t exp_addr = r.expanded + (tid & 1) * 8;
     const uint32_t sm_addr = r.sm + 8 * tid;
     uint4* out = reinterpret_cast<uint4*>(r.out + 8 * tid);
+    [[maybe_unused]] uint32_t* out32 = reinterpret_cast<uint32_t*>(r.out) + 8 * tid;
+    [[maybe_unused]] const uint4* lo_plane = reinterpret_cast<const uint4*>(r.lo + 8 * tid);
     // Shared-memory loads are issued in batches ahead of the arithmetic that uses them (the load helpers
     // keep program order): all rank entries first, then the planes, then per half of the runs the
     // expanded high bits and the sign/mantissa bytes.
@@ -383,6 +407,11 @@ __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_lo
     for (int h = 0; h < 2; ++h) {
         uint2 hi[4];
         uint2 smv[4];
+        [[maybe_unused]] uint4 lov[4];
+        if constexpr (DT == ENEC_FP32) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) lov[q] = __ldg(lo_plane + (4 * h + q) * (kBlockElems / 8 / 8));
+        }
         if constexpr (HB > 0) {
 #pragma unroll
             for (int q = 0; q < 4; ++q) hi[q] = lds64(exp_addr + rk[4 * h + q] * 16);
@@ -413,7 +442,7 @@ __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_lo
                 x1 = (r.c4_or_h - (v.y & ~Hm)) ^ ((r.c4 ^ ~v.y) & Hm);
             }
             uint32_t lo0, lo1, hi0, hi1;
-            if (DT == ENEC_BF16) {
+            if (DT != ENEC_FP16) {
                 hi0 = (smv[q].x & Hm) | ((x0 >> 1) & ~Hm);
                 hi1 = (smv[q].y & Hm) | ((x1 >> 1) & ~Hm);
                 lo0 = ((x0 << 7) & Hm) | (smv[q].x & ~Hm);
@@ -431,7 +460,8 @@ __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_lo
             w.y = prmt(lo0, hi0, 0x7362u);
             w.z = prmt(lo1, hi1, 0x5140u);
             w.w = prmt(lo1, hi1, 0x7362u);
-            out[c * (kBlockElems / 8 / 8)] = w;
+            if constexpr (DT == ENEC_FP32) store_fp32_run(out32 + c * (kBlockElems / 8), w, lov[q]);
+            else out[c * (kBlockElems / 8 / 8)] = w;
         }
     }
 }
@@ -565,6 +595,7 @@ struct BlockDesc {
     StageLayout L;
     uint16_t* out;        // global: first element of the block
     const uint8_t* high;  // global: first record of the block
+    const uint16_t* lo;   // global, fp32 only: low halves of the block's elements
 };
 static_assert(sizeof(BlockDesc) <= kStageMetaBytes, "descriptor fits the stage's meta area");
 
@@ -711,7 +742,16 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             d->b = uint32_t(jc.b);
             d->n = uint32_t(jc.n);
             d->L = L;
-            d->out = jc.out + uint64_t(k) * kBlockElems;
+            d->out = jc.out + uint64_t(k) * kBlockElems * (DT == ENEC_FP32 ? 2 : 1);
+            if (DT == ENEC_FP32) {
+                // the low halves go from global memory straight to the consumers' registers: start them
+                // towards L2 along with the block's copies
+                const uint8_t* lo = jc.in + jc.off_smlo + uint64_t(k) * kBlockElems * 2;
+                d->lo = reinterpret_cast<const uint16_t*>(lo);
+                bulk_prefetch_l2(lo, uint32_t(align16(uint64_t(real) * 2)));
+            } else {
+                d->lo = nullptr;
+            }
             d->high = jc.in + h0;
             mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes);
             bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
@@ -781,6 +821,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             r.expanded = st + o_exp;
             r.out = d->out;
             r.high = d->high;
+            r.lo = d->lo;
             r.real = d->real;
         }
         if (consumer_barrier_or(*abort_flag != 0)) break;
@@ -794,7 +835,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
 #undef ENEC_CASE
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
-        if constexpr (DTV == ENEC_BF16) {                                                    \
+        if constexpr (DTV != ENEC_FP16) {                                                    \
             if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid); \
             else decode_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, N, tid);              \
         }                                                                                    \

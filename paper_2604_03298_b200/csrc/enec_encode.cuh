@@ -73,8 +73,9 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p) {
 // ---------------------------------------------------------------------------------------------------
 template <int DT>
 struct HistShape {
-    static constexpr int E = DT == ENEC_BF16 ? 8 : 5;
+    static constexpr int E = DT == ENEC_FP16 ? 5 : 8;
     static constexpr int kBins = 1 << E;
+    static constexpr int kPerLoad = DT == ENEC_FP32 ? 4 : 8;  // values in a 16-byte load
     static constexpr int kCopies = 8;                    // copies of the histogram per warp
     static constexpr int kWarpBytes = kBins * kCopies * 4;
 };
@@ -87,8 +88,10 @@ __device__ __forceinline__ void red_add_one(uint32_t addr) {
 
 template <int DT>
 __device__ __forceinline__ void count_word_pair(uint32_t base, uint32_t w) {
-    // two 16-bit values per 32-bit word; bin x sits at byte x * 32 of the warp's area
-    if (DT == ENEC_BF16) {
+    // two 16-bit values per 32-bit word (one fp32 value); bin x sits at byte x * 32 of the warp's area
+    if (DT == ENEC_FP32) {
+        red_add_one(base + ((w >> 18) & 0x1FE0u));   // x = bits 30..23
+    } else if (DT == ENEC_BF16) {
         red_add_one(base + ((w >> 2) & 0x1FE0u));    // x = bits 14..7
         red_add_one(base + ((w >> 18) & 0x1FE0u));
     } else {
@@ -202,7 +205,8 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     cta_hist[tid] = 0;
     __syncthreads();
 
-    const uint64_t nchunks = count >> 3;  // 16-byte loads of eight values
+    constexpr int kPerLoad = HistShape<DT>::kPerLoad;
+    const uint64_t nchunks = count / kPerLoad;  // 16-byte loads of eight 16-bit or four 32-bit values
     const uint4* in4 = reinterpret_cast<const uint4*>(in);
     // a warp takes 2 KB at a time: four 16-byte loads per lane in flight before any counting
     constexpr uint32_t kUnroll = 4;
@@ -239,10 +243,13 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
         cta_hist[tid] = sum;
     }
     __syncthreads();
-    if (blockIdx.x == 0 && tid == 0) {  // the last count mod 8 values
+    if (blockIdx.x == 0 && tid == 0) {  // the values behind the last whole 16-byte load
         constexpr int sh = DT == ENEC_BF16 ? 7 : 10;
-        for (uint64_t e = nchunks << 3; e < count; ++e)
-            atomicAdd(&cta_hist[(in[e] >> sh) & (HistShape<DT>::kBins - 1)], 1u);
+        for (uint64_t e = nchunks * kPerLoad; e < count; ++e) {
+            const uint32_t x = DT == ENEC_FP32 ? (reinterpret_cast<const uint32_t*>(in)[e] >> 23) & 0xFFu
+                                               : (uint32_t(in[e]) >> sh) & (HistShape<DT>::kBins - 1);
+            atomicAdd(&cta_hist[x], 1u);
+        }
     }
     __syncthreads();
     if (cta_hist[tid]) atomicAdd(&ctl->hist[tid], (unsigned long long)cta_hist[tid]);
@@ -428,7 +435,7 @@ __device__ __forceinline__ Split4 split4(uint32_t w0, uint32_t w1) {
     const uint32_t lo = prmt(w0, w1, 0x6420u);  // low bytes of the four 16-bit words
     const uint32_t hi = prmt(w0, w1, 0x7531u);  // high bytes
     Split4 s;
-    if (DT == ENEC_BF16) {
+    if (DT != ENEC_FP16) {
         s.x = ((hi << 1) & 0xFEFEFEFEu) | ((lo >> 7) & 0x01010101u);
         s.sm = (hi & 0x80808080u) | (lo & 0x7F7F7F7Fu);
         s.hs = 0;
@@ -472,20 +479,36 @@ struct EncodeShared {
     uint32_t tainted;      // the block or a predecessor saw parameters that lose exponents
 };
 
+// fp32: the eight values at `p` (32 bytes, 16-byte aligned) as their high halves, which have bf16's layout; the
+// low halves go to `lo_dst` (16 bytes) as they are.
+__device__ __forceinline__ uint4 load_fp32_run(const uint8_t* p, uint8_t* lo_dst) {
+    const uint4 a0 = __ldcs(reinterpret_cast<const uint4*>(p));
+    const uint4 a1 = __ldcs(reinterpret_cast<const uint4*>(p) + 1);
+    __stcs(reinterpret_cast<uint4*>(lo_dst), make_uint4(prmt(a0.x, a0.y, 0x5410u), prmt(a0.z, a0.w, 0x5410u),
+                                                        prmt(a1.x, a1.y, 0x5410u), prmt(a1.z, a1.w, 0x5410u)));
+    return make_uint4(prmt(a0.x, a0.y, 0x7632u), prmt(a0.z, a0.w, 0x7632u), prmt(a1.x, a1.y, 0x7632u),
+                      prmt(a1.z, a1.w, 0x7632u));
+}
+
 // Phase 1 of a full block (16384 real elements), all 256 threads: loads, split, transform, sign/mantissa
 // stores and group widths with immediate offsets and no bounds logic. Lanes l and l + 16 share a group, so
 // the two halves of a ballot OR into the mask of the warp's sixteen groups of run c.
 // SIMPLE (n < 8 and no loss check): only the low seven bits of b - x matter, so the exponent is taken
 // without its top bit and a guard bit absorbs the borrow: y = ((b & 127 | 128) - (x & 127)) & (2^n - 1).
 // Returns the wide flags of the thread's eight runs (bit c).
+// With DT = ENEC_FP32 the values are 32-bit words: their high halves take bf16's path, their low halves are
+// stored as they are to `lo_thread` (two bytes per value).
 template <int DT, bool SIMPLE>
-__device__ __forceinline__ uint32_t encode_full_runs(const uint16_t* in_thread, uint8_t* sm_thread, const TransformCtx& tc,
-                                                     int m, uint32_t warp, uint32_t lane, uint32_t* mask_words,
-                                                     uint2 (&y)[8], uint2 (&hs)[8], int& bad) {
+__device__ __forceinline__ uint32_t encode_full_runs(const uint8_t* in_thread, uint8_t* sm_thread, uint8_t* lo_thread,
+                                                     const TransformCtx& tc, int m, uint32_t warp, uint32_t lane,
+                                                     uint32_t* mask_words, uint2 (&y)[8], uint2 (&hs)[8], int& bad) {
     constexpr uint32_t kRunStride = kBlockElems / 8;  // elements between a thread's runs
     uint4 raw[8];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) raw[c] = __ldcs(reinterpret_cast<const uint4*>(in_thread + c * kRunStride));
+    for (int c = 0; c < 8; ++c) {
+        if constexpr (DT == ENEC_FP32) raw[c] = load_fp32_run(in_thread + c * kRunStride * 4, lo_thread + c * kRunStride * 2);
+        else raw[c] = __ldcs(reinterpret_cast<const uint4*>(in_thread + c * kRunStride * 2));
+    }
     const uint32_t c7 = (tc.b4 & 0x7F7F7F7Fu) | 0x80808080u;
     const uint32_t widemask4 = ~rep4((1u << m) - 1);
     uint32_t wide_bits = 0;
@@ -496,7 +519,7 @@ __device__ __forceinline__ uint32_t encode_full_runs(const uint16_t* in_thread, 
             const uint32_t lo0 = prmt(raw[c].x, raw[c].y, 0x6420u), hi0 = prmt(raw[c].x, raw[c].y, 0x7531u);
             const uint32_t lo1 = prmt(raw[c].z, raw[c].w, 0x6420u), hi1 = prmt(raw[c].z, raw[c].w, 0x7531u);
             uint32_t x0, x1;  // exponent fields without bit 7
-            if (DT == ENEC_BF16) {
+            if (DT != ENEC_FP16) {
                 x0 = ((hi0 << 1) & 0x7E7E7E7Eu) | ((lo0 >> 7) & 0x01010101u);
                 x1 = ((hi1 << 1) & 0x7E7E7E7Eu) | ((lo1 >> 7) & 0x01010101u);
                 sm0 = (hi0 & 0x80808080u) | (lo0 & 0x7F7F7F7Fu);
@@ -535,7 +558,7 @@ __device__ __forceinline__ uint32_t encode_full_runs(const uint16_t* in_thread, 
 template <int DT>
 __device__ __noinline__ int encode_short_block(const uint16_t* in, uint32_t N, uint32_t real, const TransformCtx& tc,
                                                int b, int n, int m, int check, uint8_t* out_sm, uint8_t* out_low,
-                                               uint8_t* out_smhi, uint8_t* out_mask, EncodeShared* sh,
+                                               uint8_t* out_smhi, uint8_t* out_mask, uint8_t* out_smlo, EncodeShared* sh,
                                                uint32_t* s_low, uint32_t* s_hi3, uint32_t* s_rec) {
     const uint32_t tid = threadIdx.x;
     const int hbits = n - m;
@@ -547,9 +570,17 @@ __device__ __noinline__ int encode_short_block(const uint16_t* in, uint32_t N, u
     int bad = 0;
     uint32_t y = 0;
     if (tid < N) {
-        const uint32_t w = tid < real ? in[tid] : 0;
+        uint32_t w = 0;
+        if (DT == ENEC_FP32) {
+            // the high half goes on as a bf16 word; the low half is stored as it is (zeros pad the plane to 16 bytes)
+            const uint32_t full = tid < real ? reinterpret_cast<const uint32_t*>(in)[tid] : 0;
+            w = full >> 16;
+            if (2 * tid < uint32_t(align16(2 * real))) reinterpret_cast<uint16_t*>(out_smlo)[tid] = uint16_t(full);
+        } else if (tid < real) {
+            w = in[tid];
+        }
         uint32_t x, sm, hs = 0;
-        if (DT == ENEC_BF16) { x = (w >> 7) & 0xFF; sm = ((w >> 8) & 0x80) | (w & 0x7F); }
+        if (DT != ENEC_FP16) { x = (w >> 7) & 0xFF; sm = ((w >> 8) & 0x80) | (w & 0x7F); }
         else { x = (w >> 10) & 0x1F; sm = w & 0xFF; hs = ((w >> 13) & 4) | ((w >> 8) & 3); }
         if (tid < real) {
             y = uint32_t(b - int(x)) & ((1u << n) - 1);
@@ -742,7 +773,7 @@ __device__ __forceinline__ void resolve_block(const EncodeJob& job, const Encode
 template <int DT>
 __global__ void __launch_bounds__(kEncodeThreads, 4)
 enec_encode_kernel(EncodeJob job, int* status) {
-    constexpr int E = DT == ENEC_BF16 ? 8 : 5;
+    constexpr int E = DT == ENEC_FP16 ? 5 : 8;
     // dynamic shared memory: low plane | fp16 sign/mantissa-high plane | two record buffers
     extern __shared__ __align__(16) uint8_t enc_smem[];
     uint8_t* s_low = enc_smem;                                   // normalised bytes of the low plane
@@ -790,7 +821,10 @@ enec_encode_kernel(EncodeJob job, int* status) {
     const bool last = k + 1 == g.nblocks;
     const uint32_t N = last ? g.tail_padded : kBlockElems;
     const uint32_t real = last ? g.tail_real : kBlockElems;
-    const uint16_t* in = job.in + uint64_t(k) * kBlockElems;
+    constexpr uint32_t kElemBytes = DT == ENEC_FP32 ? 4 : 2;
+    const uint8_t* in_bytes = reinterpret_cast<const uint8_t*>(job.in) + uint64_t(k) * kBlockElems * kElemBytes;
+    const uint16_t* in = reinterpret_cast<const uint16_t*>(in_bytes);
+    uint8_t* out_smlo = job.out + sec.smlo + uint64_t(k) * kBlockElems * 2;  // fp32 only
     uint8_t* out_sm = job.out + sec.sm + uint64_t(k) * kBlockElems;
     uint8_t* out_low = job.out + sec.low + uint64_t(k) * (kBlockElems / 8) * uint32_t(m);
     uint8_t* out_smhi = job.out + sec.smhi + uint64_t(k) * (kBlockElems / 8) * 3;
@@ -811,9 +845,9 @@ enec_encode_kernel(EncodeJob job, int* status) {
     uint2 hs[8];
     if (fast) {
         if (!job.check && n < 8)
-            wide_bits = encode_full_runs<DT, true>(in + j, out_sm + j, tc, m, warp, lane, sh.mask, y, hs, bad);
+            wide_bits = encode_full_runs<DT, true>(in_bytes + j * kElemBytes, out_sm + j, out_smlo + j * 2, tc, m, warp, lane, sh.mask, y, hs, bad);
         else
-            wide_bits = encode_full_runs<DT, false>(in + j, out_sm + j, tc, m, warp, lane, sh.mask, y, hs, bad);
+            wide_bits = encode_full_runs<DT, false>(in_bytes + j * kElemBytes, out_sm + j, out_smlo + j * 2, tc, m, warp, lane, sh.mask, y, hs, bad);
         uint2 ylow[8];
         const uint32_t lowmask4 = rep4((1u << m) - 1);
 #pragma unroll
@@ -830,11 +864,27 @@ enec_encode_kernel(EncodeJob job, int* status) {
             raw[c] = make_uint4(0, 0, 0, 0);
             if (active) {
                 if (e0 + 8 <= real) {
-                    raw[c] = __ldcs(reinterpret_cast<const uint4*>(in + e0));
+                    if constexpr (DT == ENEC_FP32) raw[c] = load_fp32_run(in_bytes + e0 * 4, out_smlo + e0 * 2);
+                    else raw[c] = __ldcs(reinterpret_cast<const uint4*>(in + e0));
                 } else if (e0 < real) {
                     uint32_t v[4] = {0, 0, 0, 0};
-                    for (uint32_t i = 0; e0 + i < real; ++i) v[i >> 1] |= uint32_t(in[e0 + i]) << (16 * (i & 1));
+                    for (uint32_t i = 0; e0 + i < real; ++i) {
+                        uint32_t half;  // the 16-bit word that takes the exponent path
+                        if constexpr (DT == ENEC_FP32) {
+                            const uint32_t full = reinterpret_cast<const uint32_t*>(in_bytes)[e0 + i];
+                            reinterpret_cast<uint16_t*>(out_smlo)[e0 + i] = uint16_t(full);
+                            half = full >> 16;
+                        } else {
+                            half = in[e0 + i];
+                        }
+                        v[i >> 1] |= half << (16 * (i & 1));
+                    }
                     raw[c] = make_uint4(v[0], v[1], v[2], v[3]);
+                }
+                if constexpr (DT == ENEC_FP32) {  // zeros up to the plane's 16-byte boundary
+                    for (uint32_t i = 0; i < 8; ++i)
+                        if (e0 + i >= real && 2 * (e0 + i) < uint32_t(align16(2 * real)))
+                            reinterpret_cast<uint16_t*>(out_smlo)[e0 + i] = 0;
                 }
             }
         }
@@ -887,19 +937,23 @@ enec_encode_kernel(EncodeJob job, int* status) {
             if (DT == ENEC_FP16) pack_plane<3>(smem_u32(s_hi3), j, N, hs);
         }
     } else {
-        bad = encode_short_block<DT>(in, N, real, tc, b, n, m, job.check, out_sm, out_low, out_smhi, out_mask, &sh,
+        bad = encode_short_block<DT>(in, N, real, tc, b, n, m, job.check, out_sm, out_low, out_smhi, out_mask, out_smlo, &sh,
                                      reinterpret_cast<uint32_t*>(s_low), reinterpret_cast<uint32_t*>(s_hi3),
                                      reinterpret_cast<uint32_t*>(s_rec));
     }
     const int any_bad = __syncthreads_or(bad);
     {
-        // the CTA's next block is known by now: pull its 32 KB towards L2 (one 128-byte line per thread)
+        // the CTA's next block is known by now: pull its 32 KB towards L2 (one 128-byte line per thread, two for fp32)
         // so that the loads of the next iteration do not wait for DRAM
         const uint32_t next_block = sh.next[(iter + 1) & 1];
         if (next_block < g.nblocks) {
-            const uint8_t* line = reinterpret_cast<const uint8_t*>(job.in + uint64_t(next_block) * kBlockElems) + tid * 128;
-            const uint8_t* end = reinterpret_cast<const uint8_t*>(job.in + job.count);
-            if (line < end) asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
+            const uint8_t* base = reinterpret_cast<const uint8_t*>(job.in);
+            const uint8_t* end = base + job.count * kElemBytes;
+#pragma unroll
+            for (uint32_t r = 0; r < kElemBytes / 2; ++r) {
+                const uint8_t* line = base + uint64_t(next_block) * kBlockElems * kElemBytes + (r * kEncodeThreads + tid) * 128;
+                if (line < end) asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
+            }
         }
     }
 

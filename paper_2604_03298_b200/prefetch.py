@@ -13,7 +13,7 @@ import torch
 
 from . import binding as enec
 
-_DT = {torch.bfloat16: enec.BF16, torch.float16: enec.FP16}
+_DT = {torch.bfloat16: enec.BF16, torch.float16: enec.FP16, torch.float32: enec.FP32}
 
 
 class LayerPrefetcher:

@@ -11,7 +11,7 @@ import torch
 
 from . import binding as enec
 
-_DT = {torch.bfloat16: enec.BF16, torch.float16: enec.FP16}
+_DT = {torch.bfloat16: enec.BF16, torch.float16: enec.FP16, torch.float32: enec.FP32}
 
 
 def shard(items: list, rank: int, world: int) -> list:
@@ -70,7 +70,7 @@ class CodecSet:
 
     @property
     def raw_bytes(self) -> int:
-        return sum(t.numel() * 2 for t in self.raw)
+        return sum(t.numel() * t.element_size() for t in self.raw)
 
     def compress_all(self, params=None) -> None:
         """One enec_compress per tensor on the current stream (no host synchronisation)."""
@@ -105,5 +105,6 @@ class CodecSet:
     def verify_roundtrip(self) -> None:
         """Outputs must equal the raw tensors bit for bit (needs unshared outputs)."""
         for i, t in enumerate(self.raw):
-            if not torch.equal(self.outs[i].view(torch.int16), t.reshape(-1).view(torch.int16)):
+            bits = torch.int32 if t.element_size() == 4 else torch.int16
+            if not torch.equal(self.outs[i].view(bits), t.reshape(-1).view(bits)):
                 raise AssertionError(f"tensor {i}: decompressed bits differ from the input")

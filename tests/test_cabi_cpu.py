@@ -37,10 +37,10 @@ def test_max_compressed_size_matches_oracle(libenec, oracle):
     f = libenec.enec_max_compressed_size
     f.argtypes = [ctypes.c_int, ctypes.c_size_t]
     f.restype = ctypes.c_size_t
-    for dt in (0, 1):
+    for dt in (0, 1, 2):
         for count in (0, 1, 15, 16, 17, 4096, 16383, 16384, 16385, 123457, 1 << 20, 128256 * 4096, (1 << 36) - 1):
             assert f(dt, count) == oracle.max_compressed_size(dt, count)
-    assert f(2, 100) == 0 and f(0, 1 << 36) == 0
+    assert f(3, 100) == 0 and f(0, 1 << 36) == 0
 
 
 def test_binding_has_the_same_names():
