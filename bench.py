@@ -27,10 +27,25 @@ WORKLOADS = {
     "llama8b": (3, "full 32-layer Llama-3-8B-shaped bf16 weight set, 291 tensors, 16.06 GB"),
     "layer": (2, "one Llama-3-8B-shaped decoder layer in bf16, 9 tensors, 436 MB"),
     "tensor": (1, "one bf16 tensor 1024x4096, 8 MB"),
+    "olmo1b_fp32": (6, "OLMo-1B-shaped fp32 weight set, 115 tensors, 5.1 GB (side measurement: Sec. 6.2 fp32 support)"),
 }
 SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
+
+
+def _dtype_codes():
+    import torch
+    return {torch.bfloat16: 0, torch.float16: 1, torch.float32: 2}
+
+
+class _LazyCodes(dict):
+    def __missing__(self, key):
+        self.update(_dtype_codes())
+        return dict.__getitem__(self, key)
+
+
+DTYPE_CODE = _LazyCodes()   # torch dtype -> enec_dtype (filled on first use: torch is imported late)
 
 
 def measured_peak_gbs():
@@ -91,6 +106,15 @@ class ClockSampler:
         return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def host_words(t):
+    """Raw bit patterns of a tensor as a flat numpy array on the host (uint16, or uint32 for fp32)."""
+    import numpy as np
+    import torch
+    if t.element_size() == 4:
+        return t.reshape(-1).view(torch.int32).cpu().numpy().view(np.uint32)
+    return t.reshape(-1).view(torch.int16).cpu().numpy().view(np.uint16)
+
+
 def oracle_module():
     sys.path.insert(0, os.path.join(ROOT, "oracle"))
     import enec_oracle
@@ -99,7 +123,7 @@ def oracle_module():
 
 
 def time_oracle(words_list, dt=0):
-    """Single-threaded oracle over a list of numpy uint16 arrays. Returns (compress s, decompress s, raw bytes,
+    """Single-threaded oracle over a list of numpy arrays of raw words (uint16, or uint32 for fp32). Returns (compress s, decompress s, raw bytes,
     stream bytes)."""
     oracle = oracle_module()
     tc = td = 0.0
@@ -131,13 +155,14 @@ def run_reference(args):
     specs = synth.config_specs(cfg)
     big = [s for s in specs if s.numel >= 1 << 20]
     sample = [s for s in big if s.name.split(".")[-1] in ("q", "k", "v", "o")][:4] or big[:1]
-    words = [synth.as_words(synth.make_tensor(s, "cpu")).numpy().view(np.uint16) for s in sample]
+    words = [host_words(synth.make_tensor(s, "cpu")) for s in sample]
+    dt = DTYPE_CODE[sample[0].dtype]
     for _ in range(args.warmup):
-        time_oracle(words[:1])
+        time_oracle(words[:1], dt)
     t_comp = t_dec = 0.0
     t_all0 = time.perf_counter()
     for _ in range(args.steps):
-        tc, td, raw, comp = time_oracle(words)
+        tc, td, raw, comp = time_oracle(words, dt)
         t_comp += tc
         t_dec += td
     t_all = time.perf_counter() - t_all0
@@ -238,14 +263,14 @@ def run_ours(args):
     for h, i in zip(h_raw, layer):
         h.copy_(cs.raw[i].reshape(-1))
     torch.cuda.synchronize()
-    e2e_raw = sum(h.numel() * 2 for h in h_raw)
+    e2e_raw = sum(h.numel() * h.element_size() for h in h_raw)
     e2e_comp = sum(h.numel() for h in h_streams)
 
     def e2e_decompress():
         for h, i in zip(h_streams, layer):
             cs.streams[i][:h.numel()].copy_(h, non_blocking=True)
-            st = enec.enec_decompress(cs.streams[i], h.numel(), 0 if cs.raw[i].dtype == torch.bfloat16 else 1,
-                                      cs.raw[i].numel(), cs.outs[i], cs.status)
+            st = enec.enec_decompress(cs.streams[i], h.numel(), DTYPE_CODE[cs.raw[i].dtype], cs.raw[i].numel(),
+                                      cs.outs[i], cs.status)
             assert st == 0
         for h, i in zip(h_raw, layer):
             h.copy_(cs.outs[i], non_blocking=True)
@@ -253,7 +278,7 @@ def run_ours(args):
     def e2e_compress():
         for h, i in zip(h_raw, layer):
             cs.outs[i].copy_(h, non_blocking=True)
-            st = enec.enec_compress(cs.outs[i], 0 if cs.raw[i].dtype == torch.bfloat16 else 1, cs.raw[i].numel(),
+            st = enec.enec_compress(cs.outs[i], DTYPE_CODE[cs.raw[i].dtype], cs.raw[i].numel(),
                                     cs.streams[i], cs.streams[i].numel(), cs.sizes[i:i + 1], cs.status)
             assert st == 0
         for h, i in zip(h_streams, layer):
@@ -273,13 +298,13 @@ def run_ours(args):
 
     # the same decompress pass as one batched launch (not part of `value`: the workload says tensor by tensor)
     sizes_host = cs.sizes.cpu().tolist()
-    bf16_idx = [i for i, t in enumerate(cs.raw) if t.dtype == torch.bfloat16]
-    batch_items = [(cs.streams[i], sizes_host[i], cs.outs[i], cs.raw[i].numel()) for i in bf16_idx]
+    one_dtype = len({t.dtype for t in cs.raw}) == 1   # a batched launch takes tensors of one dtype
+    batch_items = [(cs.streams[i], sizes_host[i], cs.outs[i], t.numel()) for i, t in enumerate(cs.raw)]
 
     def batched_pass():
-        assert enec.enec_decompress_batched(batch_items, 0, cs.status) == 0
+        assert enec.enec_decompress_batched(batch_items, DTYPE_CODE[cs.raw[0].dtype], cs.status) == 0
 
-    ms_batched = time_e2e(batched_pass) if len(bf16_idx) == len(cs.raw) else None
+    ms_batched = time_e2e(batched_pass) if one_dtype else None
     cs.check_status()
     cs.verify_roundtrip()
 
@@ -287,7 +312,7 @@ def run_ours(args):
     ms_e2e_comp = time_e2e(e2e_compress)
     cs.check_status()
     for h, i in zip(h_raw, layer):  # the host copy of the last decompress must be the tensor
-        assert torch.equal(h.view(torch.int16), cs.raw[i].reshape(-1).view(torch.int16).cpu())
+        assert (host_words(h) == host_words(cs.raw[i])).all()
 
     if rank != 0:
         if world > 1:
@@ -298,13 +323,14 @@ def run_ours(args):
     n_dec = len(cs.raw)
     dec_moved = (raw_bytes + comp_bytes)                       # algorithmic bytes of one decompress pass (this rank)
     achieved = dec_moved / (ms_dec * 1e-3) / 1e9
-    elems = raw_bytes // 2
+    elems = sum(t.numel() for t in cs.raw)
+    all_bf16 = all(t.dtype == torch.bfloat16 for t in cs.raw)   # the committed DRAM counters are bf16's
     roofline = {
         "kernel": "enec_decode_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
         "algorithmic_bytes_per_launch": dec_moved / n_dec, "launches_per_step": n_dec,
         "avg_launch_us": ms_dec * 1e3 / n_dec,
-        "traffic": DECODE_DRAM_BYTES_PER_ELEM * elems / n_dec if DECODE_DRAM_BYTES_PER_ELEM else None,
+        "traffic": DECODE_DRAM_BYTES_PER_ELEM * elems / n_dec if DECODE_DRAM_BYTES_PER_ELEM and all_bf16 else None,
         "compress": {"achieved": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9,
                      "frac": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9 / peak,
                      "note": "algorithmic bytes = read raw once + write stream; the histogram pass reads raw again"},
@@ -313,11 +339,11 @@ def run_ours(args):
     # CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1 only)
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        sample_idx = [i for i, s in enumerate(specs) if s.numel >= 1 << 20][:7]   # one layer's matrices
-        if cfg == 1:
+        sample_idx = [i for i, s in enumerate(specs) if s.numel >= 1 << 20 and s.name.startswith("l0.")][:7]
+        if not sample_idx:   # no decoder layer in the set: its first tensor
             sample_idx = [0]
-        words = [cs.raw[i].reshape(-1).view(torch.int16).cpu().numpy().view(np.uint16) for i in sample_idx]
-        tc, td, sraw, scomp = time_oracle(words)
+        words = [host_words(cs.raw[i]) for i in sample_idx]
+        tc, td, sraw, scomp = time_oracle(words, DTYPE_CODE[cs.raw[sample_idx[0]].dtype])
         gpu_sizes = [int(cs.sizes[i].item()) for i in sample_idx]
         assert sum(gpu_sizes) == scomp, "GPU and oracle stream sizes differ on the sample"
         cpu = {"value": sraw / td / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",

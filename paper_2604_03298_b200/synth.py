@@ -9,6 +9,8 @@ Five workload families (``config_specs(cfg)``):
   3  32 such layers + embedding + LM head + final norm (about 16 GB)
   4  heavy-tailed stress set: 64 fp16 + 64 bf16 4096x4096 tensors (Laplace / Student-t, outliers, zeros)
   5  many-small-tensor MoE set: 768 expert matrices + 4096 vectors of 2048
+  6  OLMo-1B-shaped fp32 set (Table 3's fp32 family): 16 layers of hidden 2048 / MLP 8192, embedding and
+     LM head of 50304 rows, about 5.1 GB
 ``scale`` divides the large matrix dimensions so CPU tests can use the same recipes at small sizes.
 """
 from dataclasses import dataclass
@@ -51,7 +53,7 @@ def _llama_layer(layer: int, seed0: int, scale: int):
 
 
 def config_specs(cfg: int, scale: int = 1):
-    """List of TensorSpec for workload family ``cfg`` (1..5)."""
+    """List of TensorSpec for workload family ``cfg`` (1..6)."""
     if cfg == 1:
         return [TensorSpec("w", torch.bfloat16, (_d(1024, scale), _d(4096, scale)), "normal", 0.0, 0.02, 0)]
     if cfg == 2:
@@ -86,11 +88,23 @@ def config_specs(cfg: int, scale: int = 1):
             specs.append(TensorSpec(f"vec{v}", torch.bfloat16, (H,), "normal", 0.0, 0.02, 5000 + idx))
             idx += 1
         return specs
+    if cfg == 6:
+        H, F, V = _d(2048, scale), _d(8192, scale), _d(50304, scale)
+        specs = [TensorSpec("embed", torch.float32, (V, H), "normal", 0.0, 0.02, 6000)]
+        for layer in range(16):
+            shapes = [("q", (H, H)), ("k", (H, H)), ("v", (H, H)), ("o", (H, H)),
+                      ("gate", (F, H)), ("up", (F, H)), ("down", (H, F))]
+            for i, (nm, shp) in enumerate(shapes):
+                specs.append(TensorSpec(f"l{layer}.{nm}", torch.float32, shp, "normal", 0.0, 1.0 / math.sqrt(shp[1]),
+                                        6010 + 10 * layer + i))
+        specs.append(TensorSpec("final_norm", torch.float32, (H,), "normal", 1.0, 0.05, 6400))
+        specs.append(TensorSpec("lm_head", torch.float32, (V, H), "normal", 0.0, 0.02, 6401))
+        return specs
     raise ValueError(f"unknown config {cfg}")
 
 
 def make_tensor(spec: TensorSpec, device="cpu") -> torch.Tensor:
-    """Draws the tensor in fp32 on ``device`` and rounds it to the spec's 16-bit dtype (nearest even)."""
+    """Draws the tensor in fp32 on ``device`` and rounds it to the spec's dtype (nearest even; fp32 stays as drawn)."""
     gen = torch.Generator(device=device)
     gen.manual_seed(spec.seed)
     n = spec.numel
