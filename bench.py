@@ -216,8 +216,8 @@ def run_ours(args):
 
     # warm-up steps, then one verified round trip (outside the timed region)
     for _ in range(max(args.warmup, 1)):
-        cs.compress_all()
-        cs.decompress_all()
+        cs.compress_all(n_streams=args.streams)
+        cs.decompress_all(n_streams=args.streams)
     torch.cuda.synchronize()
     cs.check_status()
     cs.verify_roundtrip()
@@ -236,9 +236,9 @@ def run_ours(args):
     t0 = time.perf_counter()
     for k in range(args.steps):
         ev[k][0].record()
-        cs.compress_all()
+        cs.compress_all(n_streams=args.streams)
         ev[k][1].record()
-        cs.decompress_all()
+        cs.decompress_all(n_streams=args.streams)
         ev[k][2].record()
     barrier()
     wall_ms = (time.perf_counter() - t0) * 1e3
@@ -305,6 +305,9 @@ def run_ours(args):
         assert enec.enec_decompress_batched(batch_items, DTYPE_CODE[cs.raw[0].dtype], cs.status) == 0
 
     ms_batched = time_e2e(batched_pass) if one_dtype else None
+    # the two passes on one stream, for comparison with the multi-stream step
+    ms_dec_1s = time_e2e(cs.decompress_all) if args.streams > 1 else ms_dec
+    ms_comp_1s = time_e2e(cs.compress_all) if args.streams > 1 else ms_comp
     cs.check_status()
     cs.verify_roundtrip()
 
@@ -330,6 +333,7 @@ def run_ours(args):
         "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
         "algorithmic_bytes_per_launch": dec_moved / n_dec, "launches_per_step": n_dec,
         "avg_launch_us": ms_dec * 1e3 / n_dec,
+        "avg_launch_note": "duration of the decompress pass / its launches (launches of different streams overlap)",
         "traffic": DECODE_DRAM_BYTES_PER_ELEM * elems / n_dec if DECODE_DRAM_BYTES_PER_ELEM and all_bf16 else None,
         "compress": {"achieved": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9,
                      "frac": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9 / peak,
@@ -355,7 +359,11 @@ def run_ours(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": desc, "tensors_per_rank": n_dec, "raw_bytes_per_rank": raw_bytes,
-                   "step": "enec_compress of every tensor, then enec_decompress of every tensor, one stream",
+                   "step": "enec_compress of every tensor, then enec_decompress of every tensor; tensor i on side "
+                           f"stream i mod {args.streams}, forked from and joined to the timed stream with events"
+                           if args.streams > 1 else
+                           "enec_compress of every tensor, then enec_decompress of every tensor, one stream",
+                   "streams": args.streams,
                    "value_is": "uncompressed bytes / time of the step's decompress pass",
                    "l2": "inputs larger than L2 (each pass streams the whole set)" if raw_bytes > 256e6 else
                          "set fits in L2: HBM fraction not meaningful",
@@ -363,6 +371,9 @@ def run_ours(args):
         "ms_decompress_per_step": ms_dec, "ms_compress_per_step": ms_comp, "wall_ms_per_step": wall_ms / args.steps,
         "compress": {"value": total_raw / (ms_comp * 1e-3) / 1e9, "unit": "GB/s"},
         "roundtrip": {"value": total_raw / (ms_step * 1e-3) / 1e9, "unit": "GB/s"},
+        "single_stream": {"decompress": {"value": total_raw / (ms_dec_1s * 1e-3) / 1e9, "unit": "GB/s"},
+                          "compress": {"value": total_raw / (ms_comp_1s * 1e-3) / 1e9, "unit": "GB/s"},
+                          "note": "the same two passes with every call on one stream"},
         "decompress_batched": None if ms_batched is None else {
             "value": total_raw / (ms_batched * 1e-3) / 1e9, "unit": "GB/s", "launches_per_pass": 1,
             "note": "same streams through enec_decompress_batched, one launch for the whole set"},
@@ -384,10 +395,10 @@ def run_ours(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per element of enec_decode_kernel from the committed ncu capture
-# (profiles/decode_kernel_llama_layer.md: 85.55 MB read + 64.49 MB written for the 58,720,256 elements of
+# (profiles/decode_kernel_llama_layer.md: 85.54 MB read + 61.83 MB written for the 58,720,256 elements of
 # gate_proj). Below the algorithmic 3.475 B/element because part of the output is still dirty in L2 when the
 # kernel ends. Set to None when the kernel changes until a new capture exists.
-DECODE_DRAM_BYTES_PER_ELEM = (85.546496e6 + 64.491520e6) / 58720256
+DECODE_DRAM_BYTES_PER_ELEM = (85.538048e6 + 61.829120e6) / 58720256
 
 
 def main():
@@ -397,6 +408,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b", choices=sorted(WORKLOADS))
+    ap.add_argument("--streams", type=int, default=8,
+                    help="side streams the per-tensor calls of a pass are spread over (1 = everything on one stream)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

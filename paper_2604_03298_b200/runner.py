@@ -51,6 +51,8 @@ class CodecSet:
     outs: List[torch.Tensor] = field(default_factory=list)
     sizes: Optional[torch.Tensor] = None      # int64 [n]: stream lengths, written by the device
     status: Optional[torch.Tensor] = None     # int32 [1]: first device error of any call
+    shared_outs: bool = False
+    side: List[torch.cuda.Stream] = field(default_factory=list)   # side streams of the multi-stream passes
 
     @classmethod
     def allocate(cls, raw: List[torch.Tensor], share_output: bool = False) -> "CodecSet":
@@ -58,6 +60,7 @@ class CodecSet:
         cs = cls(raw=[t.contiguous() for t in raw])
         cs.streams = [torch.empty(enec.enec_max_compressed_size(_DT[t.dtype], t.numel()), dtype=torch.uint8, device=dev)
                       for t in cs.raw]
+        cs.shared_outs = share_output
         if share_output:
             biggest = max(t.numel() for t in cs.raw)
             pool = {dt: torch.empty(biggest, dtype=dt, device=dev) for dt in {t.dtype for t in cs.raw}}
@@ -72,27 +75,62 @@ class CodecSet:
     def raw_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in self.raw)
 
-    def compress_all(self, params=None) -> None:
-        """One enec_compress per tensor on the current stream (no host synchronisation)."""
-        for i, t in enumerate(self.raw):
-            dt = _DT[t.dtype]
-            if params is None:
-                st = enec.enec_compress(t, dt, t.numel(), self.streams[i], self.streams[i].numel(),
-                                        self.sizes[i:i + 1], self.status)
-            else:
-                st = enec.enec_compress_with_params(t, dt, t.numel(), *params, self.streams[i],
-                                                    self.streams[i].numel(), self.sizes[i:i + 1], self.status)
-            if st != 0:
-                raise enec.EnecError(st, f"enec_compress tensor {i}")
+    def _spread(self, n_streams: int, call) -> None:
+        """Runs call(i) for every tensor. With n_streams > 1 tensor i is enqueued on side stream i % n_streams:
+        the tensors are independent, so the start of one launch may overlap the end of another. The side
+        streams start after everything enqueued so far on the current stream, and the current stream
+        continues after all of them (events; no host synchronisation)."""
+        if n_streams > 1 and self.shared_outs:
+            raise ValueError("outputs that share one buffer cannot be written from several streams")
+        if n_streams <= 1:
+            for i in range(len(self.raw)):
+                call(i)
+            return
+        main = torch.cuda.current_stream()
+        while len(self.side) < n_streams:
+            self.side.append(torch.cuda.Stream(device=self.raw[0].device))
+        side = self.side[:n_streams]
+        start = torch.cuda.Event()
+        start.record(main)
+        for s in side:
+            s.wait_event(start)
+        for i in range(len(self.raw)):
+            with torch.cuda.stream(side[i % n_streams]):
+                call(i)
+        for s in side:
+            done = torch.cuda.Event()
+            done.record(s)
+            main.wait_event(done)
 
-    def decompress_all(self) -> None:
-        """One enec_decompress per tensor on the current stream. The stream length passed is the buffer's
-        capacity; the true length is in the stream header and is checked against it on the device."""
-        for i, t in enumerate(self.raw):
-            st = enec.enec_decompress(self.streams[i], self.streams[i].numel(), _DT[t.dtype], t.numel(),
-                                      self.outs[i], self.status)
-            if st != 0:
-                raise enec.EnecError(st, f"enec_decompress tensor {i}")
+    def compress_all(self, params=None, n_streams: int = 1) -> None:
+        """One enec_compress per tensor (no host synchronisation), on the current stream or spread over
+        n_streams side streams."""
+        self._spread(n_streams, lambda i: self._compress_one(i, params))
+
+    def _compress_one(self, i: int, params) -> None:
+        t = self.raw[i]
+        dt = _DT[t.dtype]
+        if params is None:
+            st = enec.enec_compress(t, dt, t.numel(), self.streams[i], self.streams[i].numel(),
+                                    self.sizes[i:i + 1], self.status)
+        else:
+            st = enec.enec_compress_with_params(t, dt, t.numel(), *params, self.streams[i],
+                                                self.streams[i].numel(), self.sizes[i:i + 1], self.status)
+        if st != 0:
+            raise enec.EnecError(st, f"enec_compress tensor {i}")
+
+    def decompress_all(self, n_streams: int = 1) -> None:
+        """One enec_decompress per tensor, on the current stream or spread over n_streams side streams. The
+        stream length passed is the buffer's capacity; the true length is in the stream header and is checked
+        against it on the device."""
+        self._spread(n_streams, self._decompress_one)
+
+    def _decompress_one(self, i: int) -> None:
+        t = self.raw[i]
+        st = enec.enec_decompress(self.streams[i], self.streams[i].numel(), _DT[t.dtype], t.numel(),
+                                  self.outs[i], self.status)
+        if st != 0:
+            raise enec.EnecError(st, f"enec_decompress tensor {i}")
 
     def check_status(self) -> None:
         code = int(self.status.item())
