@@ -75,15 +75,16 @@ class CodecSet:
     def raw_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in self.raw)
 
-    def _spread(self, n_streams: int, call) -> None:
-        """Runs call(i) for every tensor. With n_streams > 1 tensor i is enqueued on side stream i % n_streams:
+    def spread(self, n_streams: int, call, count: Optional[int] = None) -> None:
+        """Runs call(i) for i < count (default: for every tensor). With n_streams > 1 tensor i is enqueued on side stream i % n_streams:
         the tensors are independent, so the start of one launch may overlap the end of another. The side
         streams start after everything enqueued so far on the current stream, and the current stream
         continues after all of them (events; no host synchronisation)."""
         if n_streams > 1 and self.shared_outs:
             raise ValueError("outputs that share one buffer cannot be written from several streams")
+        count = len(self.raw) if count is None else count
         if n_streams <= 1:
-            for i in range(len(self.raw)):
+            for i in range(count):
                 call(i)
             return
         main = torch.cuda.current_stream()
@@ -94,7 +95,7 @@ class CodecSet:
         start.record(main)
         for s in side:
             s.wait_event(start)
-        for i in range(len(self.raw)):
+        for i in range(count):
             with torch.cuda.stream(side[i % n_streams]):
                 call(i)
         for s in side:
@@ -105,7 +106,7 @@ class CodecSet:
     def compress_all(self, params=None, n_streams: int = 1) -> None:
         """One enec_compress per tensor (no host synchronisation), on the current stream or spread over
         n_streams side streams."""
-        self._spread(n_streams, lambda i: self._compress_one(i, params))
+        self.spread(n_streams, lambda i: self._compress_one(i, params))
 
     def _compress_one(self, i: int, params) -> None:
         t = self.raw[i]
@@ -123,7 +124,7 @@ class CodecSet:
         """One enec_decompress per tensor, on the current stream or spread over n_streams side streams. The
         stream length passed is the buffer's capacity; the true length is in the stream header and is checked
         against it on the device."""
-        self._spread(n_streams, self._decompress_one)
+        self.spread(n_streams, self._decompress_one)
 
     def _decompress_one(self, i: int) -> None:
         t = self.raw[i]
