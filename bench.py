@@ -27,6 +27,7 @@ WORKLOADS = {
     "llama8b": (3, "full 32-layer Llama-3-8B-shaped bf16 weight set, 291 tensors, 16.06 GB"),
     "layer": (2, "one Llama-3-8B-shaped decoder layer in bf16, 9 tensors, 436 MB"),
     "tensor": (1, "one bf16 tensor 1024x4096, 8 MB"),
+    "layer_fp32": (7, "one OLMo-1B-shaped decoder layer in fp32, 7 tensors, 268 MB (side measurement)"),
     "olmo1b_fp32": (6, "OLMo-1B-shaped fp32 weight set, 115 tensors, 5.1 GB (side measurement: Sec. 6.2 fp32 support)"),
 }
 SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"

@@ -273,13 +273,22 @@ __device__ __noinline__ uint2 record_half_from_global(const uint8_t* rp, uint32_
     return second_half ? make_uint2(v.z, v.w) : make_uint2(v.x, v.y);
 }
 
-// fp32: joins the high halves of eight values (w, element order) with their low halves and stores 32 bytes.
+// fp32: joins the high halves of eight values (w, element order) with their low halves and stores 32 bytes:
+// as one 32-byte store where the address allows it, so that consecutive lanes fill whole sectors.
 __device__ __forceinline__ void store_fp32_run(uint32_t* out, uint4 w, uint4 lo) {
-    uint4* o = reinterpret_cast<uint4*>(out);
-    o[0] = make_uint4(prmt(lo.x, w.x, 0x5410u), prmt(lo.x, w.x, 0x7632u), prmt(lo.y, w.y, 0x5410u),
+    const uint4 a = make_uint4(prmt(lo.x, w.x, 0x5410u), prmt(lo.x, w.x, 0x7632u), prmt(lo.y, w.y, 0x5410u),
                       prmt(lo.y, w.y, 0x7632u));
-    o[1] = make_uint4(prmt(lo.z, w.z, 0x5410u), prmt(lo.z, w.z, 0x7632u), prmt(lo.w, w.w, 0x5410u),
+    const uint4 b = make_uint4(prmt(lo.z, w.z, 0x5410u), prmt(lo.z, w.z, 0x7632u), prmt(lo.w, w.w, 0x5410u),
                       prmt(lo.w, w.w, 0x7632u));
+    if ((reinterpret_cast<uintptr_t>(out) & 31) == 0) {
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(out), "r"(a.x), "r"(a.y), "r"(a.z),
+                     "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                     : "memory");
+    } else {
+        uint4* o = reinterpret_cast<uint4*>(out);
+        o[0] = a;
+        o[1] = b;
+    }
 }
 
 // Finishes eight consecutive elements e0 .. e0+7 of a block: high bits of wide groups, inverse transform,

@@ -481,9 +481,17 @@ struct EncodeShared {
 
 // fp32: the eight values at `p` (32 bytes, 16-byte aligned) as their high halves, which have bf16's layout; the
 // low halves go to `lo_dst` (16 bytes) as they are.
-__device__ __forceinline__ uint4 load_fp32_run(const uint8_t* p, uint8_t* lo_dst) {
-    const uint4 a0 = __ldcs(reinterpret_cast<const uint4*>(p));
-    const uint4 a1 = __ldcs(reinterpret_cast<const uint4*>(p) + 1);
+__device__ __forceinline__ uint4 load_fp32_run(const uint8_t* __restrict__ p, uint8_t* __restrict__ lo_dst) {
+    uint4 a0, a1;
+    if ((reinterpret_cast<uintptr_t>(p) & 31) == 0) {
+        // one 32-byte load: consecutive lanes read consecutive 32-byte pieces
+        asm("ld.global.cs.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+            : "=r"(a0.x), "=r"(a0.y), "=r"(a0.z), "=r"(a0.w), "=r"(a1.x), "=r"(a1.y), "=r"(a1.z), "=r"(a1.w)
+            : "l"(p));
+    } else {
+        a0 = __ldcs(reinterpret_cast<const uint4*>(p));
+        a1 = __ldcs(reinterpret_cast<const uint4*>(p) + 1);
+    }
     __stcs(reinterpret_cast<uint4*>(lo_dst), make_uint4(prmt(a0.x, a0.y, 0x5410u), prmt(a0.z, a0.w, 0x5410u),
                                                         prmt(a1.x, a1.y, 0x5410u), prmt(a1.z, a1.w, 0x5410u)));
     return make_uint4(prmt(a0.x, a0.y, 0x7632u), prmt(a0.z, a0.w, 0x7632u), prmt(a1.x, a1.y, 0x7632u),

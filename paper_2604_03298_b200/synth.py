@@ -11,6 +11,7 @@ Five workload families (``config_specs(cfg)``):
   5  many-small-tensor MoE set: 768 expert matrices + 4096 vectors of 2048
   6  OLMo-1B-shaped fp32 set (Table 3's fp32 family): 16 layers of hidden 2048 / MLP 8192, embedding and
      LM head of 50304 rows, about 5.1 GB
+  7  one decoder layer of family 6 (seven fp32 matrices, 268 MB)
 ``scale`` divides the large matrix dimensions so CPU tests can use the same recipes at small sizes.
 """
 from dataclasses import dataclass
@@ -53,7 +54,7 @@ def _llama_layer(layer: int, seed0: int, scale: int):
 
 
 def config_specs(cfg: int, scale: int = 1):
-    """List of TensorSpec for workload family ``cfg`` (1..6)."""
+    """List of TensorSpec for workload family ``cfg`` (1..7)."""
     if cfg == 1:
         return [TensorSpec("w", torch.bfloat16, (_d(1024, scale), _d(4096, scale)), "normal", 0.0, 0.02, 0)]
     if cfg == 2:
@@ -88,17 +89,18 @@ def config_specs(cfg: int, scale: int = 1):
             specs.append(TensorSpec(f"vec{v}", torch.bfloat16, (H,), "normal", 0.0, 0.02, 5000 + idx))
             idx += 1
         return specs
-    if cfg == 6:
+    if cfg in (6, 7):
         H, F, V = _d(2048, scale), _d(8192, scale), _d(50304, scale)
-        specs = [TensorSpec("embed", torch.float32, (V, H), "normal", 0.0, 0.02, 6000)]
-        for layer in range(16):
+        specs = [TensorSpec("embed", torch.float32, (V, H), "normal", 0.0, 0.02, 6000)] if cfg == 6 else []
+        for layer in range(16 if cfg == 6 else 1):
             shapes = [("q", (H, H)), ("k", (H, H)), ("v", (H, H)), ("o", (H, H)),
                       ("gate", (F, H)), ("up", (F, H)), ("down", (H, F))]
             for i, (nm, shp) in enumerate(shapes):
                 specs.append(TensorSpec(f"l{layer}.{nm}", torch.float32, shp, "normal", 0.0, 1.0 / math.sqrt(shp[1]),
                                         6010 + 10 * layer + i))
-        specs.append(TensorSpec("final_norm", torch.float32, (H,), "normal", 1.0, 0.05, 6400))
-        specs.append(TensorSpec("lm_head", torch.float32, (V, H), "normal", 0.0, 0.02, 6401))
+        if cfg == 6:
+            specs.append(TensorSpec("final_norm", torch.float32, (H,), "normal", 1.0, 0.05, 6400))
+            specs.append(TensorSpec("lm_head", torch.float32, (V, H), "normal", 0.0, 0.02, 6401))
         return specs
     raise ValueError(f"unknown config {cfg}")
 

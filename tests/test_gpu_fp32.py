@@ -170,3 +170,31 @@ def test_ratio_of_gaussian_weights(oracle):
     assert 1.12 < ratio < 1.20
     back = enec.decompress_tensor(stream, torch.float32, t.shape)
     assert torch.equal(back.view(torch.int32).cpu(), t.view(torch.int32))
+
+
+def test_buffers_on_odd_sixteen_byte_boundaries(oracle):
+    """Input and output that start 16 bytes behind a 32-byte boundary take the paths with 16-byte accesses."""
+    import paper_2604_03298_b200 as enec
+    count = 16384 * 5 + 300
+    w = gaussian_words(count, 31)
+    want = oracle.compress(w, FP32)
+    holder = torch.zeros(count + 4, dtype=torch.float32, device="cuda")
+    assert holder.data_ptr() % 32 == 0
+    d_in = holder[4:]
+    d_in.copy_(dev_words(w))
+    cap = enec.enec_max_compressed_size(FP32, count)
+    buf = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    size = torch.zeros(1, dtype=torch.int64, device="cuda")
+    status = status_tensor()
+    assert enec.enec_compress(d_in, FP32, count, buf, cap, size, status) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = buf[:int(size.item())].cpu().numpy()
+    assert np.array_equal(got, want)
+    out_holder = torch.full((count + 8,), 7.0, dtype=torch.float32, device="cuda")
+    out = out_holder[4:4 + count]
+    assert enec.enec_decompress(buf, cap, FP32, count, out, status) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(host_words(out), w)
+    assert (out_holder[:4] == 7.0).all() and (out_holder[4 + count:] == 7.0).all()
