@@ -208,29 +208,42 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     constexpr int kPerLoad = HistShape<DT>::kPerLoad;
     const uint64_t nchunks = count / kPerLoad;  // 16-byte loads of eight 16-bit or four 32-bit values
     const uint4* in4 = reinterpret_cast<const uint4*>(in);
-    // a warp takes 2 KB at a time: four 16-byte loads per lane in flight before any counting
+    // a warp takes 2 KB at a time (four 16-byte loads per lane) and asks for its next 2 KB before it counts
+    // the ones it holds, so four to eight loads per lane are in flight all the time
     constexpr uint32_t kUnroll = 4;
-    const uint64_t warps_total = uint64_t(gridDim.x) * (kHistThreads / 32);
-    for (uint64_t first = (uint64_t(blockIdx.x) * (kHistThreads / 32) + warp) * (32 * kUnroll); first < nchunks;
-         first += warps_total * (32 * kUnroll)) {
-        uint4 v[kUnroll];
+    const uint64_t stride = uint64_t(gridDim.x) * (kHistThreads / 32) * (32 * kUnroll);
+    uint64_t first = (uint64_t(blockIdx.x) * (kHistThreads / 32) + warp) * (32 * kUnroll);
+    uint4 cur[kUnroll], nxt[kUnroll];
+    // back to front, default caching: the encode pass reads the tensor again from the front, where the lines
+    // touched last are the likeliest to be in L2 still
+    auto load = [&](uint4 (&v)[kUnroll], uint64_t at) {
 #pragma unroll
         for (uint32_t u = 0; u < kUnroll; ++u) {
-            const uint64_t i = first + u * 32 + lane;
+            const uint64_t i = at + u * 32 + lane;
             v[u] = make_uint4(0, 0, 0, 0);
-            // back to front, default caching: the encode pass reads the tensor again from the front, where
-            // the lines touched last are the likeliest to be in L2 still
             if (i < nchunks) v[u] = in4[nchunks - 1 - i];
         }
+    };
+    auto count4 = [&](const uint4 (&v)[kUnroll], uint64_t at) {
 #pragma unroll
         for (uint32_t u = 0; u < kUnroll; ++u) {
-            if (first + u * 32 + lane < nchunks) {
+            if (at + u * 32 + lane < nchunks) {
                 count_word_pair<DT>(base, v[u].x);
                 count_word_pair<DT>(base, v[u].y);
                 count_word_pair<DT>(base, v[u].z);
                 count_word_pair<DT>(base, v[u].w);
             }
         }
+    };
+    if (first < nchunks) load(cur, first);
+    while (first < nchunks) {
+        load(nxt, first + stride);
+        count4(cur, first);
+        first += stride;
+        if (first >= nchunks) break;
+        load(cur, first + stride);
+        count4(nxt, first);
+        first += stride;
     }
     __syncthreads();
     if (tid < uint32_t(HistShape<DT>::kBins)) {  // fold the warps' copies of bin `tid`

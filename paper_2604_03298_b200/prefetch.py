@@ -66,6 +66,18 @@ class LayerPrefetcher:
             self.freed[b].record(main)
         main.wait_stream(self.side)
 
+    def capture(self, forward: Callable[[int, List[torch.Tensor]], None], overlap: bool = True) -> "torch.cuda.CUDAGraph":
+        """Records one run() (all layers: decompress launches, the events between the two streams and whatever
+        `forward` enqueues) into a CUDA graph and returns it; `graph.replay()` then repeats the whole pass with
+        one submission. A layer's batched launch carries its tensor list in the kernel parameters, so the
+        recorded launches need no descriptor copy. `forward` must not synchronise with the host."""
+        self.run(forward, overlap)          # first use outside the capture: module attributes, allocator warm-up
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(forward, overlap)
+        return graph
+
     def check_status(self) -> None:
         code = int(self.status.item())
         if code != 0:

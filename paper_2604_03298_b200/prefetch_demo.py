@@ -1,6 +1,7 @@
 """Measures what layer-wise decompression costs a forward pass on one GPU: Llama-3-8B-shaped layers, GEMMs of
 `tokens` rows against every weight matrix, (a) weights resident uncompressed, (b) each layer decompressed on the
-same stream right before use, (c) the next layer decompressed on a side stream meanwhile. Prints one JSON line.
+same stream right before use, (c) the next layer decompressed on a side stream meanwhile, (d) pass (c) recorded
+into a CUDA graph and replayed. Prints one JSON line.
 
     python -m paper_2604_03298_b200.prefetch_demo [--layers 8] [--tokens 2048] [--steps 10]
 """
@@ -57,6 +58,8 @@ def main():
     ms_serial = timed(lambda: pf.run(forward, overlap=False))
     ms_overlap = timed(lambda: pf.run(forward, overlap=True))
     ms_decode_only = timed(lambda: pf.run(lambda i, w: None, overlap=False))
+    graph = pf.capture(forward, overlap=True)
+    ms_graph = timed(graph.replay)
     pf.check_status()
     flops = 2.0 * args.tokens * sum(w.numel() for w in raw_layers[0]) * args.layers
     raw_bytes = sum(w.numel() * 2 for layer in raw_layers for w in layer)
@@ -65,7 +68,8 @@ def main():
         "layers": args.layers, "tokens": args.tokens, "steps": args.steps,
         "weights_raw_bytes": raw_bytes, "weights_compressed_bytes": comp_bytes,
         "ms_forward_resident": ms_resident, "ms_forward_decompress_same_stream": ms_serial,
-        "ms_forward_prefetch_side_stream": ms_overlap, "ms_decompress_only": ms_decode_only,
+        "ms_forward_prefetch_side_stream": ms_overlap, "ms_forward_prefetch_cuda_graph": ms_graph,
+        "ms_decompress_only": ms_decode_only,
         "gemm_tflops_resident": flops / (ms_resident * 1e-3) / 1e12,
         "overlap_cost_ms": ms_overlap - ms_resident, "serial_cost_ms": ms_serial - ms_resident,
         "hidden_fraction_of_decompress": 1.0 - (ms_overlap - ms_resident) / ms_decode_only,

@@ -47,3 +47,31 @@ def test_prefetched_layers_are_bit_exact(overlap):
     pf.check_status()
     assert seen == list(range(len(layers))) * 3
     assert int(sink.sum().item()) == 0
+
+
+def test_a_captured_pass_replays_bit_exact():
+    """The whole prefetched pass recorded into a CUDA graph: every replay decompresses every layer again."""
+    from paper_2604_03298_b200.prefetch import LayerPrefetcher
+    raw_layers, layers = _compressed_layers(n_layers=5, scale=8)
+    pf = LayerPrefetcher(layers, torch.bfloat16)
+    sink = torch.zeros(len(layers), dtype=torch.int64, device="cuda")
+    scratch = [torch.zeros_like(w, dtype=torch.bool) for w in raw_layers[0]]
+
+    def forward(i, weights):
+        total = sink[i] * 0
+        for w, r, tmp in zip(weights, raw_layers[i], scratch):
+            torch.ne(w.view(torch.int16), r.view(torch.int16), out=tmp)
+            total = total + tmp.sum()
+        sink[i] += total + 1       # one per visit, plus the number of differing words
+
+    graph = pf.capture(forward)
+    torch.cuda.synchronize()
+    sink.zero_()
+    for rep in range(3):
+        for buf in pf.buffers:     # a replay must not pass on what an earlier pass left in the buffers
+            for t in buf:
+                t.zero_()
+        graph.replay()
+    torch.cuda.synchronize()
+    pf.check_status()
+    assert sink.tolist() == [3] * len(layers)
