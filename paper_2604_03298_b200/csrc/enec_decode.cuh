@@ -621,6 +621,62 @@ struct DecodeBatch {
     uint32_t inline_prefix[kInlineJobs + 1];
 };
 
+// 16 bytes from global memory through L2 only (no copy is left in L1, which is not coherent).
+__device__ __forceinline__ uint4 ldg_l2_only(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Runs before the wait on the previous kernel of the stream, one thread per CTA: asks L2 for the
+// compressed bytes of the CTA's first blocks, so that the copies issued after the wait find them there.
+// What it reads may still be about to be written by that previous kernel, so nothing read here is
+// used for anything but prefetch addresses, every address stays inside the caller's buffer
+// [in, in + in_size), and the loads bypass L1; L2 is coherent, so a line prefetched too early is simply
+// updated by the writer. Only for tensor lists that travel in the kernel parameters.
+template <int DT>
+__device__ __forceinline__ void prefetch_before_wait(const DecodeBatch& batch, uint32_t first_block, uint32_t n_mine) {
+    if (batch.jobs != nullptr || n_mine == 0) return;
+    uint32_t j = 0;
+    while (j + 1 < batch.n_jobs && batch.inline_prefix[j + 1] <= first_block) ++j;
+    const DecodeJob& job = batch.inline_jobs[j];
+    const uint32_t k = first_block - batch.inline_prefix[j];
+    if (job.in_size < kHeaderBytes + 4 * (uint64_t(k) + 3) + 16) return;
+    const uint4 h0 = ldg_l2_only(job.in);        // magic, version/dtype, count
+    const uint4 h1 = ldg_l2_only(job.in + 16);   // block, b/n/m/L, nblocks, total_groups
+    const uint4 h2 = ldg_l2_only(job.in + 32);   // a_total
+    const int n = int((h1.y >> 8) & 0xFF), m = int((h1.y >> 16) & 0xFF);
+    if (h0.x != kMagic || n < 1 || n > exp_bits(DT) || m < 1 || m > n) return;
+    const Geometry g = make_geometry(job.count);
+    if (k >= g.nblocks) return;
+    const Sections sec = make_sections(DT, job.count, g, n, m, h2.x);
+    if (sec.total > job.in_size) return;
+    const uint32_t* table = reinterpret_cast<const uint32_t*>(job.in + sec.table);
+    const uint32_t ahead = n_mine < kStages ? n_mine : kStages;
+    for (uint32_t i = 0; i < ahead && k + i < g.nblocks; ++i) {
+        const uint32_t kk = k + i;
+        const bool tail = kk + 1 == g.nblocks;
+        const uint32_t N = tail ? g.tail_padded : kBlockElems;
+        const uint32_t real = tail ? g.tail_real : kBlockElems;
+        uint32_t t0, t1;
+        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(t0) : "l"(table + kk));
+        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(t1) : "l"(table + kk + 1));
+        bulk_prefetch_l2(job.in + sec.mask + uint64_t(kk) * (kGroupsPerBlock / 8), uint32_t(align16(((N >> 4) + 7) / 8)));
+        bulk_prefetch_l2(job.in + sec.low + uint64_t(kk) * (kBlockElems / 8) * m, uint32_t(align16(uint64_t(N) * m / 8)));
+        if (DT == ENEC_FP16)
+            bulk_prefetch_l2(job.in + sec.smhi + uint64_t(kk) * (kBlockElems / 8) * 3, uint32_t(align16(uint64_t(N) * 3 / 8)));
+        bulk_prefetch_l2(job.in + sec.sm + uint64_t(kk) * kBlockElems, uint32_t(align16(real)));
+        if (DT == ENEC_FP32)
+            bulk_prefetch_l2(job.in + sec.smlo + uint64_t(kk) * kBlockElems * 2, uint32_t(align16(uint64_t(real) * 2)));
+        const uint32_t hbits = uint32_t(n - m);
+        if (hbits > 0 && t1 > t0 && t1 - t0 <= (N >> 4)) {
+            const uint64_t r0 = (sec.high + uint64_t(t0) * 2 * hbits) & ~uint64_t(15);
+            const uint64_t r1 = align16(sec.high + uint64_t(t1) * 2 * hbits);
+            if (r1 <= sec.total && r1 > r0) bulk_prefetch_l2(job.in + r0, uint32_t(r1 - r0));
+        }
+    }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
 enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
@@ -630,15 +686,11 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     constexpr uint32_t S = kStages;
 
     pdl_launch_dependents();
-    pdl_wait();  // nothing above touches global memory
-    if (batch.total_blocks == 0) {  // nothing to decode: only check the header of a single empty tensor
-        if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr && batch.n_jobs == 1) {
-            JobCtx jc;
-            const int err = load_job<DT>(batch.inline_jobs[0], jc);
-            if (err) report(status, err);
-        }
-        return;
-    }
+    // everything up to pdl_wait() may run while the previous kernel of the stream still does
+    const uint32_t first_block = uint32_t(uint64_t(blockIdx.x) * batch.total_blocks / gridDim.x);
+    const uint32_t end_block = uint32_t(uint64_t(blockIdx.x + 1) * batch.total_blocks / gridDim.x);
+    const uint32_t n_mine = end_block - first_block;
+    if (threadIdx.x == kConsumerWarps * 32) prefetch_before_wait<DT>(batch, first_block, n_mine);
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(&ctl->full[s], 1);
@@ -648,13 +700,19 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
         mbar_fence_init();
     }
     __syncthreads();
+    pdl_wait();  // nothing above uses what it read from global memory, except as prefetch addresses
+    if (batch.total_blocks == 0) {  // nothing to decode: only check the header of a single empty tensor
+        if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr && batch.n_jobs == 1) {
+            JobCtx jc;
+            const int err = load_job<DT>(batch.inline_jobs[0], jc);
+            if (err) report(status, err);
+        }
+        return;
+    }
 
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lane = threadIdx.x & 31;
     volatile int* abort_flag = &ctl->abort;
-    const uint32_t first_block = uint32_t(uint64_t(blockIdx.x) * batch.total_blocks / gridDim.x);
-    const uint32_t end_block = uint32_t(uint64_t(blockIdx.x + 1) * batch.total_blocks / gridDim.x);
-    const uint32_t n_mine = end_block - first_block;
 
     if (warp == kConsumerWarps) {
         // ---------------- loader warp: lane 0 issues the copies of block after block ----------------

@@ -1,6 +1,6 @@
 """The five workload families at their full sizes, through the calls and launch configuration the benchmark times
-(runner.CodecSet: one enec_compress and one enec_decompress per tensor, spread over eight side streams as in the
-benchmark's default, and on one stream).
+(runner.CodecSet: one enec_compress and one enec_decompress per tensor on one stream; the Llama set also with the
+calls spread over eight side streams, as in the benchmark's multi-stream measurement).
 
 Every tensor must come back bit for bit (tolerance 0). Every stream must be self-consistent (header length = the
 length the device reported, within the bound of enec_max_compressed_size). A sample of tensors that the CPU oracle
@@ -12,10 +12,10 @@ import torch
 pytestmark = pytest.mark.gpu
 
 
-BENCH_STREAMS = 8   # bench.py's default
+SPREAD_STREAMS = 8   # bench.py's --spread-streams default
 
 
-def _run_set(specs, oracle, sample, reuse=None, n_streams=BENCH_STREAMS):
+def _run_set(specs, oracle, sample, reuse=None, n_streams=1):
     import paper_2604_03298_b200 as enec
     from paper_2604_03298_b200 import runner, synth
     cache = {}
@@ -61,7 +61,7 @@ def test_config2_llama_layer_full(oracle):
     assert 1.36 < ratio < 1.40
 
 
-@pytest.mark.parametrize("n_streams", [BENCH_STREAMS, 1])
+@pytest.mark.parametrize("n_streams", [1, SPREAD_STREAMS])
 def test_config3_llama8b_full(oracle, n_streams):
     from paper_2604_03298_b200 import synth
     specs = synth.config_specs(3)
