@@ -35,18 +35,9 @@ SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.acti
              "clocks_event_reasons.sw_power_cap")
 
 
-def _dtype_codes():
-    import torch
-    return {torch.bfloat16: 0, torch.float16: 1, torch.float32: 2}
-
-
-class _LazyCodes(dict):
-    def __missing__(self, key):
-        self.update(_dtype_codes())
-        return dict.__getitem__(self, key)
-
-
-DTYPE_CODE = _LazyCodes()   # torch dtype -> enec_dtype (filled on first use: torch is imported late)
+def dtype_code(dtype):
+    """enec_dtype of a torch dtype."""
+    return {"torch.bfloat16": 0, "torch.float16": 1, "torch.float32": 2}[str(dtype)]
 
 
 def measured_peak_gbs():
@@ -157,7 +148,7 @@ def run_reference(args):
     big = [s for s in specs if s.numel >= 1 << 20]
     sample = [s for s in big if s.name.split(".")[-1] in ("q", "k", "v", "o")][:4] or big[:1]
     words = [host_words(synth.make_tensor(s, "cpu")) for s in sample]
-    dt = DTYPE_CODE[sample[0].dtype]
+    dt = dtype_code(sample[0].dtype)
     for _ in range(args.warmup):
         time_oracle(words[:1], dt)
     t_comp = t_dec = 0.0
@@ -272,7 +263,7 @@ def run_ours(args):
     def e2e_decompress_one(j):
         i, h_in, h_out = layer[j], h_streams[j], h_raw[j]
         cs.streams[i][:h_in.numel()].copy_(h_in, non_blocking=True)
-        st = enec.enec_decompress(cs.streams[i], h_in.numel(), DTYPE_CODE[cs.raw[i].dtype], cs.raw[i].numel(),
+        st = enec.enec_decompress(cs.streams[i], h_in.numel(), dtype_code(cs.raw[i].dtype), cs.raw[i].numel(),
                                   cs.outs[i], cs.status)
         assert st == 0
         h_out.copy_(cs.outs[i], non_blocking=True)
@@ -280,7 +271,7 @@ def run_ours(args):
     def e2e_compress_one(j):
         i, h_in, h_out = layer[j], h_raw[j], h_streams[j]
         cs.outs[i].copy_(h_in, non_blocking=True)
-        st = enec.enec_compress(cs.outs[i], DTYPE_CODE[cs.raw[i].dtype], cs.raw[i].numel(),
+        st = enec.enec_compress(cs.outs[i], dtype_code(cs.raw[i].dtype), cs.raw[i].numel(),
                                 cs.streams[i], cs.streams[i].numel(), cs.sizes[i:i + 1], cs.status)
         assert st == 0
         h_out.copy_(cs.streams[i][:h_out.numel()], non_blocking=True)
@@ -309,7 +300,7 @@ def run_ours(args):
     batch_items = [(cs.streams[i], sizes_host[i], cs.outs[i], t.numel()) for i, t in enumerate(cs.raw)]
 
     def batched_pass():
-        assert enec.enec_decompress_batched(batch_items, DTYPE_CODE[cs.raw[0].dtype], cs.status) == 0
+        assert enec.enec_decompress_batched(batch_items, dtype_code(cs.raw[0].dtype), cs.status) == 0
 
     ms_batched = time_e2e(batched_pass) if one_dtype else None
     # the same steps again with the calls spread over several streams (the timed step itself keeps the
@@ -367,7 +358,7 @@ def run_ours(args):
         if not sample_idx:   # no decoder layer in the set: its first tensor
             sample_idx = [0]
         words = [host_words(cs.raw[i]) for i in sample_idx]
-        tc, td, sraw, scomp = time_oracle(words, DTYPE_CODE[cs.raw[sample_idx[0]].dtype])
+        tc, td, sraw, scomp = time_oracle(words, dtype_code(cs.raw[sample_idx[0]].dtype))
         gpu_sizes = [int(cs.sizes[i].item()) for i in sample_idx]
         assert sum(gpu_sizes) == scomp, "GPU and oracle stream sizes differ on the sample"
         cpu = {"value": sraw / td / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
