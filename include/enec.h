@@ -21,6 +21,10 @@
  *
  * The library keeps one small device scratch area per (device, stream) for the compressor (histogram
  * and control words); it is allocated on the first compress call on that stream and kept until exit.
+ * The area carries state from one compress call on the stream to the next (that is what saves clearing it
+ * every call), so: compress calls on ONE stream are issued by one host thread at a time, and
+ * enec_compress / enec_compress_with_params on a stream that is being captured into a CUDA graph return
+ * ENEC_ERR_INVALID_ARG (a replay would not see the state). Decompression keeps no state and can be captured.
  */
 #ifndef ENEC_H
 #define ENEC_H

@@ -73,25 +73,67 @@ static enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaSt
 struct ScratchArea {
     uint8_t* ptr = nullptr;
     size_t bytes = 0;
+    uint32_t epoch = 0;       // compressor areas: number of the last call
+    bool needs_clear = true;  // compressor areas: fresh memory, a wrapped epoch or a launch that failed
 };
 
 enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1 };
 
-static enec_status get_scratch(int dev, cudaStream_t stream, ScratchKind kind, size_t need, uint8_t** out) {
-    static std::mutex mu;
+static std::mutex g_scratch_mu;
+static ScratchArea& scratch_area(int dev, cudaStream_t stream, ScratchKind kind) {
     static std::map<std::pair<std::pair<int, int>, cudaStream_t>, ScratchArea> areas;
-    std::lock_guard<std::mutex> lock(mu);
-    ScratchArea& a = areas[std::make_pair(std::make_pair(dev, int(kind)), stream)];
-    if (a.bytes < need) {
-        size_t bytes = a.bytes ? a.bytes : size_t(64) << 10;
-        while (bytes < need) bytes *= 2;
-        void* p = nullptr;
-        if (cudaMalloc(&p, bytes) != cudaSuccess) return ENEC_ERR_CUDA;
-        a.ptr = static_cast<uint8_t*>(p);
-        a.bytes = bytes;
+    return areas[std::make_pair(std::make_pair(dev, int(kind)), stream)];
+}
+
+static enec_status grow(ScratchArea& a, size_t need) {
+    if (a.bytes >= need) return ENEC_OK;
+    size_t bytes = a.bytes ? a.bytes : size_t(64) << 10;
+    while (bytes < need) bytes *= 2;
+    void* p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) return ENEC_ERR_CUDA;
+    a.ptr = static_cast<uint8_t*>(p);
+    a.bytes = bytes;
+    a.needs_clear = true;
+    return ENEC_OK;
+}
+
+static enec_status get_scratch(int dev, cudaStream_t stream, ScratchKind kind, size_t need, uint8_t** out) {
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    ScratchArea& a = scratch_area(dev, stream, kind);
+    const enec_status st = grow(a, need);
+    *out = a.ptr;
+    return st;
+}
+
+// Scratch of one compress call and the call's number on it. The area is cleared (on `stream`) only when it
+// is new, when the numbers have run out or after a call on it failed to launch; otherwise the kernels keep
+// it usable from call to call (see EncodeControl).
+static enec_status lease_compress_scratch(int dev, cudaStream_t stream, size_t need, uint8_t** out, uint32_t* epoch) {
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    ScratchArea& a = scratch_area(dev, stream, kScratchCompress);
+    const enec_status st = grow(a, need);
+    if (st != ENEC_OK) return st;
+    if (a.needs_clear || a.epoch >= kEpochMax) {
+        if (cudaMemsetAsync(a.ptr, 0, a.bytes, stream) != cudaSuccess) return ENEC_ERR_CUDA;
+        a.needs_clear = false;
+        a.epoch = 0;
     }
     *out = a.ptr;
+    *epoch = ++a.epoch;
     return ENEC_OK;
+}
+
+static void mark_compress_scratch_unclean(int dev, cudaStream_t stream) {
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    scratch_area(dev, stream, kScratchCompress).needs_clear = true;
+}
+
+// The job's pointers into a scratch area for call number `epoch`.
+static void place_job(EncodeJob& job, uint8_t* scratch, uint32_t epoch) {
+    job.ctl = reinterpret_cast<EncodeControl*>(scratch + (epoch & 1) * kControlSlotBytes);
+    job.ctl_next = reinterpret_cast<EncodeControl*>(scratch + ((epoch & 1) ^ 1) * kControlSlotBytes);
+    job.state = reinterpret_cast<unsigned long long*>(scratch + kControlBytes);
+    job.epoch = epoch;
 }
 
 template <int DT>
@@ -150,23 +192,28 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
     DeviceInfo& info = device_info(dev);
     const Geometry g = make_geometry(count);
     const size_t need = kControlBytes + size_t(g.nblocks) * sizeof(unsigned long long);
+    // the scratch area carries state from call to call, which a replayed recording would not see
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return ENEC_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) return ENEC_ERR_INVALID_ARG;
     uint8_t* scratch = nullptr;
-    const enec_status st = get_scratch(dev, stream, kScratchCompress, need, &scratch);
+    uint32_t epoch = 0;
+    enec_status st = lease_compress_scratch(dev, stream, need, &scratch, &epoch);
     if (st != ENEC_OK) return st;
-    if (cudaMemsetAsync(scratch, 0, need, stream) != cudaSuccess) return ENEC_ERR_CUDA;
     EncodeJob job;
     job.in = static_cast<const uint16_t*>(d_in);
     job.out = static_cast<uint8_t*>(d_out);
     job.count = count;
-    job.ctl = reinterpret_cast<EncodeControl*>(scratch);
-    job.state = reinterpret_cast<unsigned long long*>(scratch + kControlBytes);
+    place_job(job, scratch, epoch);
     job.out_size = out_size;
     job.b = b; job.n = n; job.m = m;
     job.from_search = with_params ? 0 : 1;
     job.check = with_params ? 1 : 0;
-    return dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream)
-           : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream)
-                             : launch_encode<ENEC_FP32>(job, g.nblocks, !with_params, d_status, info, stream);
+    st = dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream)
+         : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream)
+                           : launch_encode<ENEC_FP32>(job, g.nblocks, !with_params, d_status, info, stream);
+    if (st != ENEC_OK) mark_compress_scratch_unclean(dev, stream);  // a kernel of the call may not have run
+    return st;
 }
 
 // ---- compression without any allocation ------------------------------------------------------------
@@ -323,8 +370,7 @@ enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count,
     job.in = static_cast<const uint16_t*>(d_in);
     job.out = static_cast<uint8_t*>(d_out);
     job.count = count;
-    job.ctl = reinterpret_cast<EncodeControl*>(scratch);
-    job.state = reinterpret_cast<unsigned long long*>(scratch + kControlBytes);
+    place_job(job, scratch, 1);  // everything was just cleared, so every call is call number 1
     job.out_size = out_size;
     job.b = 0; job.n = 0; job.m = 0;
     job.from_search = 1;

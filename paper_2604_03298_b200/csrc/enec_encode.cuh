@@ -18,9 +18,14 @@ namespace enec {
 
 constexpr int kEncodeThreads = 256;
 constexpr int kHistThreads = 256;
-constexpr uint32_t kControlBytes = 4096;  // control area in front of the per-block state words
+constexpr uint32_t kControlSlotBytes = 4096;             // one set of control words
+constexpr uint32_t kControlBytes = 2 * kControlSlotBytes;  // control area in front of the per-block state words
 
-// Device scratch of one compress call: control words, then one 64-bit state word per block.
+// Device scratch of a compressor: two sets of control words, then one 64-bit state word per block. Nothing
+// is cleared between calls. Calls on the area are numbered (the epoch, 1 .. 2^29 - 1): call e uses control
+// set e mod 2, which it finds zeroed, and its encode kernel zeroes the other set for call e + 1 (that set's
+// last user, call e - 1, has finished before any kernel of call e reads or writes global memory). A state
+// word carries the epoch of the call that wrote it and counts as empty in every other call.
 struct alignas(16) EncodeControl {
     unsigned long long hist[256];  // exponent histogram (2^E bins used)
     uint32_t ticket;               // next block to hand out
@@ -28,21 +33,30 @@ struct alignas(16) EncodeControl {
     uint32_t reserved;
     int b, n, m;                   // result of the parameter search
 };
-static_assert(sizeof(EncodeControl) <= kControlBytes, "control area");
+static_assert(sizeof(EncodeControl) <= kControlSlotBytes, "a control set fits its slot");
 
 // state word: bits 63..62 = kind, bit 61 = this block or one summed into the value saw parameters that lose
-// exponents, bits 31..0 = value. Failure travels inside the words, so no fence is needed around them.
+// exponents, bits 60..32 = epoch of the writing call, bits 31..0 = value. Failure travels inside the words, so
+// no fence is needed around them.
 constexpr unsigned long long kStateAggregate = 1ull << 62;  // value = wide groups in the block
 constexpr unsigned long long kStatePrefix = 2ull << 62;     // value = wide groups up to and including the block
 constexpr unsigned long long kStatePoison = 3ull << 62;     // a predecessor failed
 constexpr unsigned long long kStateTaint = 1ull << 61;
+constexpr uint32_t kEpochMax = (1u << 29) - 1;
+__host__ __device__ constexpr unsigned long long epoch_bits(uint32_t epoch) { return (unsigned long long)epoch << 32; }
+// The word as this call sees it: words of other calls are empty.
+__device__ __forceinline__ unsigned long long state_of_epoch(unsigned long long word, uint32_t epoch) {
+    return (uint32_t(word >> 32) & kEpochMax) == epoch ? word : 0ull;
+}
 
 struct EncodeJob {
     const uint16_t* in;
     uint8_t* out;
     uint64_t count;
-    EncodeControl* ctl;
+    EncodeControl* ctl;            // this call's control set (zero when the call starts)
+    EncodeControl* ctl_next;       // the other set: zeroed by this call's encode kernel
     unsigned long long* state;
+    uint32_t epoch;                // number of this call on the scratch area
     unsigned long long* out_size;  // device, may be null
     int b, n, m;                   // used when from_search == 0
     int from_search;               // take (b, n, m) from ctl
@@ -196,7 +210,6 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     __shared__ int s_last;
     constexpr int kWarpBytes = HistShape<DT>::kWarpBytes;
     pdl_launch_dependents();
-    pdl_wait();  // nothing above touches global memory
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t warp_base = smem_u32(smem) + warp * kWarpBytes;
     const uint32_t base = warp_base + (lane & 7) * 4;
@@ -204,6 +217,7 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
         reinterpret_cast<uint32_t*>(smem)[i] = 0;
     cta_hist[tid] = 0;
     __syncthreads();
+    pdl_wait();  // nothing above touches global memory
 
     constexpr int kPerLoad = HistShape<DT>::kPerLoad;
     const uint64_t nchunks = count / kPerLoad;  // 16-byte loads of eight 16-bit or four 32-bit values
@@ -690,7 +704,7 @@ __device__ __forceinline__ void resolve_block(const EncodeJob& job, const Encode
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int64_t idx = pos - (i * 32 + int64_t(lane));
-                st[i] = idx >= 0 ? ld_relaxed_u64(&job.state[idx]) : kStatePrefix;
+                st[i] = idx >= 0 ? state_of_epoch(ld_relaxed_u64(&job.state[idx]), job.epoch) : kStatePrefix;
             }
             uint32_t mine = 0;      // this lane's share of the sum
             uint32_t advanced = 0;  // windows of 32 fully summed in this round
@@ -734,11 +748,11 @@ __device__ __forceinline__ void resolve_block(const EncodeJob& job, const Encode
                 sh.before = before;
                 sh.poisoned = 0;
                 sh.tainted = tainted;
-                st_relaxed_u64(&job.state[k], kStatePrefix | (tainted ? kStateTaint : 0ull) |
+                st_relaxed_u64(&job.state[k], kStatePrefix | (tainted ? kStateTaint : 0ull) | epoch_bits(job.epoch) |
                                                   (unsigned long long)(before + wide_count));
             } else {
                 if (outcome == 3) report(status, ENEC_ERR_TIMEOUT);
-                st_relaxed_u64(&job.state[k], kStatePoison);
+                st_relaxed_u64(&job.state[k], kStatePoison | epoch_bits(job.epoch));
                 sh.poisoned = 1;
                 sh.tainted = 1;
                 sh.before = 0;
@@ -805,6 +819,10 @@ enec_encode_kernel(EncodeJob job, int* status) {
     pdl_launch_dependents();
     pdl_wait();  // nothing above touches global memory
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (blockIdx.x == 0) {  // the next call on this scratch area finds its control set zeroed
+        job.ctl_next->hist[tid] = 0;
+        if (tid == 0) { job.ctl_next->ticket = 0; job.ctl_next->hist_done = 0; }
+    }
     int b = job.b, n = job.n, m = job.m;
     if (job.from_search) { b = job.ctl->b; n = job.ctl->n; m = job.ctl->m; }
     const int hbits = n - m;
@@ -992,7 +1010,8 @@ enec_encode_kernel(EncodeJob job, int* status) {
     if (tid == 31) {
         if (any_bad) report(status, ENEC_ERR_PARAMS_NOT_LOSSLESS);
         // publish this block's count at once; block 0 knows its prefix already
-        st_relaxed_u64(&job.state[k], (k == 0 ? kStatePrefix : kStateAggregate) | (any_bad ? kStateTaint : 0ull) | wide_count);
+        st_relaxed_u64(&job.state[k], (k == 0 ? kStatePrefix : kStateAggregate) | (any_bad ? kStateTaint : 0ull) |
+                                          epoch_bits(job.epoch) | wide_count);
     }
     if (N >= 128) {
         fold_plane_out(smem_u32(s_low), N * uint32_t(m) / 8, out_low, tid);
