@@ -205,3 +205,65 @@ def test_back_to_back_calls_on_one_stream(oracle):
         want = oracle.compress(words, dt)
         got = buf[:int(size.item())].cpu().numpy()
         assert np.array_equal(got, want), describe_mismatch(got, want)
+
+
+def test_scratch_state_survives_mixed_call_sequences(oracle):
+    """The compressor's scratch area is not cleared between calls: shrinking and growing tensors, both dtypes,
+    calls with and without the parameter search and a call that reports lost exponents, all queued on one stream
+    without a host synchronisation in between, must each give the oracle's stream."""
+    import paper_2604_03298_b200 as enec
+    rng = np.random.default_rng(77)
+    plan = []   # (words, dt, params or None, expect_error)
+    for rep in range(3):
+        for count in (16384 * 20 + 7, 40, 16384 * 3, 16384 * 64, 5000):
+            plan.append((_field_words(rng, count, 0, 121, 6, 3), 0, None, False))
+            plan.append((_field_words(rng, count, 1, 12, 4, 2), 1, (12, 4, 2), False))
+        lossy = (np.array([100, 130] * 9000, np.uint16) << 7).astype(np.uint16)
+        plan.append((lossy, 0, (120, 3, 2), True))
+        plan.append((_field_words(rng, 16384 * 5 + 1, 0, 124, 5, 2), 0, (124, 5, 2), False))
+    queued = []
+    for words, dt, params, _ in plan:
+        d_in = tensor_of(words, DT[dt])
+        cap = enec.enec_max_compressed_size(dt, words.size)
+        buf = torch.empty(cap, dtype=torch.uint8, device="cuda")
+        size = torch.zeros(1, dtype=torch.int64, device="cuda")
+        status = status_tensor()
+        if params is None:
+            assert enec.enec_compress(d_in, dt, words.size, buf, cap, size, status) == 0
+        else:
+            assert enec.enec_compress_with_params(d_in, dt, words.size, *params, buf, cap, size, status) == 0
+        queued.append((d_in, buf, size, status))
+    torch.cuda.synchronize()
+    for (words, dt, params, expect_error), (_, buf, size, status) in zip(plan, queued):
+        if expect_error:
+            assert int(status.item()) == -5 and int(size.item()) == 0
+            continue
+        assert int(status.item()) == 0
+        want = oracle.compress(words, dt, params)
+        got = buf[:int(size.item())].cpu().numpy()
+        assert np.array_equal(got, want), describe_mismatch(got, want)
+
+
+def test_compress_refuses_a_stream_that_is_being_captured():
+    """Compress calls keep state between calls, so they cannot be part of a CUDA graph; decompress can."""
+    import paper_2604_03298_b200 as enec
+    src = (torch.randn(16384 * 4, device="cuda") * 0.02).to(torch.bfloat16)
+    cap = enec.enec_max_compressed_size(0, src.numel())
+    dst = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    size = torch.zeros(1, dtype=torch.int64, device="cuda")
+    status = status_tensor()
+    out = torch.zeros_like(src)
+    assert enec.enec_compress(src, 0, src.numel(), dst, cap, size, status) == 0
+    assert enec.enec_decompress(dst, cap, 0, src.numel(), out, status) == 0     # first use outside a capture
+    torch.cuda.synchronize()
+    codes = {}
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        codes["compress"] = enec.enec_compress(src, 0, src.numel(), dst, cap, size, status)
+        codes["decompress"] = enec.enec_decompress(dst, cap, 0, src.numel(), out, status)
+    assert codes == {"compress": -1, "decompress": 0}
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(out.view(torch.int16), src.view(torch.int16))
