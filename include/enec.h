@@ -109,6 +109,17 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
                                     enec_stream_t stream);
 
 /*
+ * Compress n_items tensors of one dtype with two launches (the histograms and parameter searches of all
+ * tensors, then the encode of all their blocks), each tensor into a stream of its own exactly as
+ * enec_compress would write it. Entries in HOST memory: d_in = values, d_out = stream buffer, count =
+ * elements, size = capacity of d_out (at least enec_max_compressed_size(dt, count)). d_out_sizes (device
+ * array of n_items 8-byte words, may be NULL) receives the stream lengths. Meant for checkpoints made of
+ * many small tensors; the same conventions as enec_decompress_batched. Output buffers must not overlap.
+ */
+enec_status enec_compress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, size_t* d_out_sizes,
+                                  int* d_status, enec_stream_t stream);
+
+/*
  * enec_compress for callers that must not allocate device memory. (The paper has no counterpart: this is
  * a property of this library's interface, not of the codec.)
  *

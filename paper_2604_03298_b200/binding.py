@@ -50,6 +50,8 @@ def lib():
         L.enec_decompress.restype = C.c_int
         L.enec_decompress_batched.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.enec_decompress_batched.restype = C.c_int
+        L.enec_compress_batched.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.enec_compress_batched.restype = C.c_int
         L.enec_launch_count.argtypes = []
         L.enec_launch_count.restype = C.c_uint64
         L.enec_version.argtypes = []
@@ -99,6 +101,15 @@ def enec_decompress_batched(items, dt, d_status=None) -> int:
     for i, (src, nbytes, dst, count) in enumerate(items):
         arr[i].d_in, arr[i].d_out, arr[i].count, arr[i].size = src.data_ptr(), dst.data_ptr(), count, nbytes
     return lib().enec_decompress_batched(C.cast(arr, C.c_void_p), len(items), dt, _ptr(d_status), _stream())
+
+
+def enec_compress_batched(items, dt, d_out_sizes=None, d_status=None) -> int:
+    """items: list of (tensor, stream_buffer, count, capacity); d_out_sizes: int64 CUDA tensor [len(items)] or None."""
+    arr = (BatchItem * len(items))()
+    for i, (src, dst, count, capacity) in enumerate(items):
+        arr[i].d_in, arr[i].d_out, arr[i].count, arr[i].size = src.data_ptr(), dst.data_ptr(), count, capacity
+    return lib().enec_compress_batched(C.cast(arr, C.c_void_p), len(items), dt, _ptr(d_out_sizes), _ptr(d_status),
+                                       _stream())
 
 
 def enec_launch_count() -> int:

@@ -3,6 +3,7 @@
 #include <map>
 #include <mutex>
 #include <utility>
+#include <cstring>
 #include <vector>
 
 #include "enec_decode.cuh"
@@ -17,6 +18,7 @@ struct DeviceInfo {
     bool decode_attr_set[3] = {false, false, false};
     bool hist_attr_set[3] = {false, false, false};
     bool encode_attr_set[3] = {false, false, false};
+    bool batch_attr_set[3] = {false, false, false};
 };
 
 static DeviceInfo& device_info(int dev) {
@@ -77,7 +79,7 @@ struct ScratchArea {
     bool needs_clear = true;  // compressor areas: fresh memory, a wrapped epoch or a launch that failed
 };
 
-enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1 };
+enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1, kScratchCompressBatch = 2 };
 
 static std::mutex g_scratch_mu;
 static ScratchArea& scratch_area(int dev, cudaStream_t stream, ScratchKind kind) {
@@ -157,14 +159,43 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
     if (!info.encode_attr_set[DT]) {
-        if (cudaFuncSetAttribute(enec_encode_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(enec_encode_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(EncodeSmem<DT>::kBytes)) != cudaSuccess)
             return ENEC_ERR_CUDA;
         info.encode_attr_set[DT] = true;
     }
     uint32_t grid = uint32_t(info.sms) * 4;  // four resident CTAs per SM, each takes block after block
     if (grid > nblocks) grid = nblocks;
-    const cudaError_t err = launch_pdl(enec_encode_kernel<DT>, grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream, job, d_status);
+    const cudaError_t err = launch_pdl(enec_encode_kernel<DT, false>, grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream,
+                                       job, EncodeBatch{}, d_status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
+}
+
+// The two launches of a batched compress call: histograms and parameter search of every tensor, then the
+// encode of all their blocks.
+template <int DT>
+static enec_status launch_encode_batched(const EncodeJob* d_jobs, const HistUnit* d_units, uint32_t n_units,
+                                         const EncodeBatch& batch, int* d_status, DeviceInfo& info, cudaStream_t stream) {
+    const uint32_t hist_smem = HistShape<DT>::kWarpBytes * (kHistThreads / 32);
+    if (!info.batch_attr_set[DT]) {
+        if (cudaFuncSetAttribute(enec_histogram_batched_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(hist_smem)) != cudaSuccess ||
+            cudaFuncSetAttribute(enec_encode_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(EncodeSmem<DT>::kBytes)) != cudaSuccess)
+            return ENEC_ERR_CUDA;
+        info.batch_attr_set[DT] = true;
+    }
+    uint32_t grid = uint32_t(info.sms) * 3;
+    if (grid > n_units) grid = n_units;
+    if (launch_pdl(enec_histogram_batched_kernel<DT>, grid, kHistThreads, hist_smem, stream, d_jobs, d_units, n_units) !=
+        cudaSuccess)
+        return ENEC_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    grid = uint32_t(info.sms) * 4;
+    if (grid > batch.total_blocks) grid = batch.total_blocks;
+    const cudaError_t err = launch_pdl(enec_encode_kernel<DT, true>, grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream,
+                                       EncodeJob{}, batch, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
@@ -341,6 +372,91 @@ enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t co
     return compress_common(d_in, dt, count, true, b, n, m, d_out, out_capacity, d_out_size, d_status, stream);
 }
 
+
+enec_status enec_compress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, size_t* d_out_sizes,
+                                  int* d_status, enec_stream_t stream) {
+    if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if (n_items < 0 || (n_items > 0 && !h_items) || (reinterpret_cast<uintptr_t>(d_out_sizes) & 7))
+        return ENEC_ERR_INVALID_ARG;
+    if (n_items == 0) return ENEC_OK;
+    for (int i = 0; i < n_items; ++i) {
+        const enec_batch_item& it = h_items[i];
+        if ((!it.d_in && it.count) || !it.d_out || (uint64_t(it.count) >> 36) || !aligned16(it.d_in) || !aligned16(it.d_out))
+            return ENEC_ERR_INVALID_ARG;
+        if (it.size < enec_max_compressed_size(dt, it.count)) return ENEC_ERR_BUFFER_TOO_SMALL;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
+    DeviceInfo& info = device_info(dev);
+    unsigned long long* sizes = reinterpret_cast<unsigned long long*>(d_out_sizes);
+    // device scratch of the call: [ticket | control words per tensor | state word per block | jobs | prefix | units];
+    // everything in front of the tables is cleared, the tables are copied from the host
+    constexpr size_t kCtlStride = (sizeof(EncodeControl) + 63) & ~size_t(63);
+    std::vector<uint32_t> prefix(size_t(n_items) + 1);
+    std::vector<HistUnit> units;
+    uint64_t total_blocks = 0;
+    for (int i = 0; i < n_items; ++i) {
+        prefix[i] = uint32_t(total_blocks);
+        const uint64_t count = h_items[i].count;
+        if (count == 0) continue;  // written by a launch of its own below
+        total_blocks += make_geometry(count).nblocks;
+        const uint64_t chunks = (count * uint64_t(elem_bytes(dt))) >> 4;
+        const uint32_t n = chunks ? uint32_t((chunks + kHistUnitChunks - 1) / kHistUnitChunks) : 1u;
+        for (uint32_t u = 0; u < n; ++u) units.push_back(HistUnit{uint32_t(i), u, n, 0u});
+    }
+    if (total_blocks >> 32) return ENEC_ERR_INVALID_ARG;
+    prefix[n_items] = uint32_t(total_blocks);
+    const size_t off_ctl = 256;
+    const size_t off_state = (off_ctl + size_t(n_items) * kCtlStride + 255) & ~size_t(255);
+    const size_t off_jobs = (off_state + size_t(total_blocks) * sizeof(unsigned long long) + 255) & ~size_t(255);
+    const size_t off_prefix = off_jobs + size_t(n_items) * sizeof(EncodeJob);
+    const size_t off_units = (off_prefix + prefix.size() * sizeof(uint32_t) + 15) & ~size_t(15);
+    const size_t need = off_units + units.size() * sizeof(HistUnit);
+    uint8_t* scratch = nullptr;
+    const enec_status st = get_scratch(dev, stream, kScratchCompressBatch, need, &scratch);
+    if (st != ENEC_OK) return st;
+    std::vector<uint8_t> host(need - off_jobs);
+    EncodeJob* jobs = reinterpret_cast<EncodeJob*>(host.data());
+    for (int i = 0; i < n_items; ++i) {
+        EncodeJob& job = jobs[i];
+        job.in = static_cast<const uint16_t*>(h_items[i].d_in);
+        job.out = static_cast<uint8_t*>(h_items[i].d_out);
+        job.count = h_items[i].count;
+        job.ctl = reinterpret_cast<EncodeControl*>(scratch + off_ctl + size_t(i) * kCtlStride);
+        job.ctl_next = nullptr;
+        job.state = reinterpret_cast<unsigned long long*>(scratch + off_state) + prefix[i];
+        job.epoch = 1;  // the area was just cleared
+        job.out_size = sizes ? sizes + i : nullptr;
+        job.b = 0; job.n = 0; job.m = 0;
+        job.from_search = 1;
+        job.check = 0;
+    }
+    memcpy(host.data() + (off_prefix - off_jobs), prefix.data(), prefix.size() * sizeof(uint32_t));
+    if (!units.empty()) memcpy(host.data() + (off_units - off_jobs), units.data(), units.size() * sizeof(HistUnit));
+    for (int i = 0; i < n_items; ++i) {
+        if (h_items[i].count != 0) continue;
+        enec_encode_empty_kernel<<<1, 32, 0, stream>>>(static_cast<uint8_t*>(h_items[i].d_out), int(dt), 0, 1, 1,
+                                                      sizes ? sizes + i : nullptr);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return ENEC_ERR_CUDA;
+    }
+    if (total_blocks == 0) return ENEC_OK;
+    if (cudaMemsetAsync(scratch, 0, off_jobs, stream) != cudaSuccess) return ENEC_ERR_CUDA;
+    // pageable source: the call returns once the bytes are staged, so `host` may go out of scope
+    if (cudaMemcpyAsync(scratch + off_jobs, host.data(), host.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return ENEC_ERR_CUDA;
+    EncodeBatch batch;
+    batch.jobs = reinterpret_cast<const EncodeJob*>(scratch + off_jobs);
+    batch.prefix = reinterpret_cast<const uint32_t*>(scratch + off_prefix);
+    batch.n_jobs = uint32_t(n_items);
+    batch.total_blocks = uint32_t(total_blocks);
+    batch.ticket = reinterpret_cast<uint32_t*>(scratch);
+    const HistUnit* d_units = reinterpret_cast<const HistUnit*>(scratch + off_units);
+    const uint32_t n_units = uint32_t(units.size());
+    return dt == ENEC_BF16   ? launch_encode_batched<ENEC_BF16>(batch.jobs, d_units, n_units, batch, d_status, info, stream)
+           : dt == ENEC_FP16 ? launch_encode_batched<ENEC_FP16>(batch.jobs, d_units, n_units, batch, d_status, info, stream)
+                             : launch_encode_batched<ENEC_FP32>(batch.jobs, d_units, n_units, batch, d_status, info, stream);
+}
 
 enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
                                   size_t* d_out_size, int* d_status, enec_stream_t stream) {

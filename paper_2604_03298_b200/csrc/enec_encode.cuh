@@ -289,6 +289,95 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     parameter_search<DT>(ctl);
 }
 
+// Histograms of a list of tensors in one launch. The tensors are cut into units of at most kHistUnitChunks
+// 16-byte loads; a CTA takes unit after unit, adds the unit's counts to its tensor's histogram, and the CTA
+// that finishes a tensor's last outstanding unit runs that tensor's parameter search.
+constexpr uint32_t kHistUnitChunks = 16384;  // 256 KB
+struct HistUnit {
+    uint32_t job;            // tensor of the unit
+    uint32_t index;          // unit number inside the tensor
+    uint32_t units_of_job;
+    uint32_t pad;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kHistThreads, 3)
+enec_histogram_batched_kernel(const EncodeJob* __restrict__ jobs, const HistUnit* __restrict__ units, uint32_t n_units) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ uint32_t cta_hist[256];
+    __shared__ int s_last;
+    constexpr int kWarpBytes = HistShape<DT>::kWarpBytes;
+    constexpr int kPerLoad = HistShape<DT>::kPerLoad;
+    pdl_launch_dependents();
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t base = smem_u32(smem) + warp * kWarpBytes + (lane & 7) * 4;
+    for (uint32_t i = tid; i < uint32_t(kWarpBytes / 4) * (kHistThreads / 32); i += kHistThreads)
+        reinterpret_cast<uint32_t*>(smem)[i] = 0;
+    cta_hist[tid] = 0;
+    __syncthreads();
+    pdl_wait();  // nothing above touches global memory
+    for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
+        const HistUnit unit = units[u];
+        const uint16_t* in = jobs[unit.job].in;
+        const uint64_t count = jobs[unit.job].count;
+        EncodeControl* ctl = jobs[unit.job].ctl;
+        const uint64_t nchunks = count / kPerLoad;
+        const uint64_t first = uint64_t(unit.index) * kHistUnitChunks;
+        const uint64_t end = first + kHistUnitChunks < nchunks ? first + kHistUnitChunks : nchunks;
+        const uint4* in4 = reinterpret_cast<const uint4*>(in);
+        for (uint64_t at = first + tid; at < end; at += 4 * kHistThreads) {
+            uint4 v[4];
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q) {
+                v[q] = make_uint4(0, 0, 0, 0);
+                if (at + q * kHistThreads < end) v[q] = in4[at + q * kHistThreads];
+            }
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q) {
+                if (at + q * kHistThreads < end) {
+                    count_word_pair<DT>(base, v[q].x);
+                    count_word_pair<DT>(base, v[q].y);
+                    count_word_pair<DT>(base, v[q].z);
+                    count_word_pair<DT>(base, v[q].w);
+                }
+            }
+        }
+        __syncthreads();
+        if (tid < uint32_t(HistShape<DT>::kBins)) {  // fold the warps' copies of bin `tid` and clear them for the next unit
+            uint32_t sum = 0;
+            for (uint32_t wp = 0; wp < kHistThreads / 32; ++wp) {
+                const uint32_t row = smem_u32(smem) + wp * kWarpBytes + tid * 32;
+                const uint4 lo = lds128(row), hi = lds128(row + 16);
+                sum += lo.x + lo.y + lo.z + lo.w + hi.x + hi.y + hi.z + hi.w;
+                sts128(row, make_uint4(0, 0, 0, 0));
+                sts128(row + 16, make_uint4(0, 0, 0, 0));
+            }
+            cta_hist[tid] = sum;
+        }
+        __syncthreads();
+        if (tid == 0 && unit.index + 1 == unit.units_of_job) {  // the values behind the last whole 16-byte load
+            constexpr int sh = DT == ENEC_BF16 ? 7 : 10;
+            for (uint64_t e = nchunks * kPerLoad; e < count; ++e) {
+                const uint32_t x = DT == ENEC_FP32 ? (reinterpret_cast<const uint32_t*>(in)[e] >> 23) & 0xFFu
+                                                   : (uint32_t(in[e]) >> sh) & (HistShape<DT>::kBins - 1);
+                cta_hist[x] += 1;
+            }
+        }
+        __syncthreads();
+        if (cta_hist[tid]) atomicAdd(&ctl->hist[tid], (unsigned long long)cta_hist[tid]);
+        cta_hist[tid] = 0;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = atomicAdd(&ctl->hist_done, 1u) == unit.units_of_job - 1;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            parameter_search<DT>(ctl);
+        }
+        __syncthreads();
+    }
+}
+
 // ---------------------------------------------------------------------------------------------------
 // Algorithm 2 on packed bytes (forward). A thread that owns the eight lanes j..j+7 of the deepest level
 // owns, at every level, whole runs of eight consecutive lanes: the 64 elements {j + c N/8 + i : c, i < 8}.
@@ -805,10 +894,45 @@ __device__ __forceinline__ void resolve_block(const EncodeJob& job, const Encode
     }
 }
 
+// A list of tensors compressed by one launch: the blocks of all tensors form one index space that the
+// CTAs' tickets run over; every tensor keeps its own control words, state words and output.
+struct EncodeBatch {
+    const EncodeJob* jobs;   // device array [n_jobs]
+    const uint32_t* prefix;  // device array [n_jobs + 1]: blocks before each tensor
+    uint32_t n_jobs;
+    uint32_t total_blocks;
+    uint32_t* ticket;        // next block of the index space (zero when the launch starts)
+};
+
+// What a block needs to know about its tensor (batched launches keep it in shared memory per block).
+struct BlockCtx {
+    EncodeJob job;
+    EncodeTensor tensor;
+    TransformCtx tc;
+    uint32_t k;  // block index inside the tensor
+};
+
 template <int DT>
-__global__ void __launch_bounds__(kEncodeThreads, 4)
-enec_encode_kernel(EncodeJob job, int* status) {
+__device__ __forceinline__ void fill_tensor_ctx(const EncodeJob& job, EncodeTensor& tensor, TransformCtx& tc) {
     constexpr int E = DT == ENEC_FP16 ? 5 : 8;
+    int b = job.b, n = job.n, m = job.m;
+    if (job.from_search) { b = job.ctl->b; n = job.ctl->n; m = job.ctl->m; }
+    tensor.g = make_geometry(job.count);
+    tensor.sec = make_sections(DT, job.count, tensor.g, n, m, 0);
+    tensor.b = b; tensor.n = n; tensor.m = m; tensor.hbits = n - m;
+    tc.b4 = rep4(uint32_t(b));
+    tc.b4_or_h = tc.b4 | 0x80808080u;
+    tc.nmask4 = rep4((1u << n) - 1);
+    tc.s4 = rep4(1u << (n - 1));
+    tc.emask4 = rep4((1u << E) - 1);
+    tc.n = n;
+    tc.E = E;
+}
+
+// BATCH = false: one tensor, described by `single`. BATCH = true: the tensors of `batch`; `single` is unused.
+template <int DT, bool BATCH>
+__global__ void __launch_bounds__(kEncodeThreads, 4)
+enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status) {
     // dynamic shared memory: low plane | fp16 sign/mantissa-high plane | two record buffers
     extern __shared__ __align__(16) uint8_t enc_smem[];
     uint8_t* s_low = enc_smem;                                   // normalised bytes of the low plane
@@ -819,28 +943,28 @@ enec_encode_kernel(EncodeJob job, int* status) {
     pdl_launch_dependents();
     pdl_wait();  // nothing above touches global memory
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (blockIdx.x == 0) {  // the next call on this scratch area finds its control set zeroed
-        job.ctl_next->hist[tid] = 0;
-        if (tid == 0) { job.ctl_next->ticket = 0; job.ctl_next->hist_done = 0; }
+    __shared__ BlockCtx s_ctx[BATCH ? 3 : 1];  // batched: this block's, the previous block's and the next block's tensor
+    EncodeTensor single_tensor{};
+    TransformCtx single_tc{};
+    if constexpr (!BATCH) {
+        if (blockIdx.x == 0) {  // the next call on this scratch area finds its control set zeroed
+            single.ctl_next->hist[tid] = 0;
+            if (tid == 0) { single.ctl_next->ticket = 0; single.ctl_next->hist_done = 0; }
+        }
+        fill_tensor_ctx<DT>(single, single_tensor, single_tc);
     }
-    int b = job.b, n = job.n, m = job.m;
-    if (job.from_search) { b = job.ctl->b; n = job.ctl->n; m = job.ctl->m; }
-    const int hbits = n - m;
-    EncodeTensor tensor;
-    tensor.g = make_geometry(job.count);
-    tensor.sec = make_sections(DT, job.count, tensor.g, n, m, 0);
-    tensor.b = b; tensor.n = n; tensor.m = m; tensor.hbits = hbits;
-    const Geometry& g = tensor.g;
-    const Sections& sec = tensor.sec;
-
-    TransformCtx tc;
-    tc.b4 = rep4(uint32_t(b));
-    tc.b4_or_h = tc.b4 | 0x80808080u;
-    tc.nmask4 = rep4((1u << n) - 1);
-    tc.s4 = rep4(1u << (n - 1));
-    tc.emask4 = rep4((1u << E) - 1);
-    tc.n = n;
-    tc.E = E;
+    uint32_t* const ticket = BATCH ? batch.ticket : &single.ctl->ticket;
+    const uint32_t total_blocks = BATCH ? batch.total_blocks : single_tensor.g.nblocks;
+    // batched, thread 0 only: the tensor of a ticket (tickets of a CTA grow, so the search only moves forward)
+    uint32_t ctx_j = 0;
+    auto stage_ctx = [&](uint32_t ticket_value, uint32_t slot) {
+        if (ticket_value >= total_blocks) return;
+        while (batch.prefix[ctx_j + 1] <= ticket_value) ++ctx_j;
+        BlockCtx& cx = s_ctx[slot];
+        cx.job = batch.jobs[ctx_j];
+        fill_tensor_ctx<DT>(cx.job, cx.tensor, cx.tc);
+        cx.k = ticket_value - batch.prefix[ctx_j];
+    };
 
     // Persistent loop over tickets. A block's look-back is put off until the CTA has done the first half of
     // its next block: by then the predecessors, which started at about the same time, have published their
@@ -849,13 +973,27 @@ enec_encode_kernel(EncodeJob job, int* status) {
     // waits end.
     uint32_t pending_block = 0xFFFFFFFFu, pending_wide = 0, cur = 0;
     bool pending_bad = false;
-    if (tid == 0) sh.next[0] = atomicAdd(&job.ctl->ticket, 1u);
-    for (uint32_t iter = 0;; ++iter) {
+    if (tid == 0) {
+        sh.next[0] = atomicAdd(ticket, 1u);
+        if constexpr (BATCH) stage_ctx(sh.next[0], 0);
+    }
+    uint32_t iter = 0;
+    for (;; ++iter) {
     __syncthreads();
-    const uint32_t k = sh.next[iter & 1];
-    if (k >= g.nblocks) break;
+    if (sh.next[iter & 1] >= total_blocks) break;
     // the ticket after this one goes to the other slot, which nobody reads before the next barrier
-    if (tid == 0) sh.next[(iter + 1) & 1] = atomicAdd(&job.ctl->ticket, 1u);
+    if (tid == 0) {
+        sh.next[(iter + 1) & 1] = atomicAdd(ticket, 1u);
+        if constexpr (BATCH) stage_ctx(sh.next[(iter + 1) & 1], (iter + 1) % 3);
+    }
+    const BlockCtx& cx = s_ctx[BATCH ? iter % 3 : 0];
+    const EncodeJob& job = BATCH ? cx.job : single;
+    const EncodeTensor& tensor = BATCH ? cx.tensor : single_tensor;
+    const TransformCtx& tc = BATCH ? cx.tc : single_tc;
+    const Geometry& g = tensor.g;
+    const Sections& sec = tensor.sec;
+    const int b = tensor.b, n = tensor.n, m = tensor.m, hbits = tensor.hbits;
+    const uint32_t k = BATCH ? cx.k : sh.next[iter & 1];
     uint8_t* s_rec = s_rec_base + cur * EncodeSmem<DT>::kRecBytes;
     const bool last = k + 1 == g.nblocks;
     const uint32_t N = last ? g.tail_padded : kBlockElems;
@@ -984,7 +1122,7 @@ enec_encode_kernel(EncodeJob job, int* status) {
     {
         // the CTA's next block is known by now: pull its 32 KB towards L2 (one 128-byte line per thread, two for fp32)
         // so that the loads of the next iteration do not wait for DRAM
-        const uint32_t next_block = sh.next[(iter + 1) & 1];
+        const uint32_t next_block = BATCH ? 0xFFFFFFFFu : sh.next[(iter + 1) & 1];  // batched: tensors are small
         if (next_block < g.nblocks) {
             const uint8_t* base = reinterpret_cast<const uint8_t*>(job.in);
             const uint8_t* end = base + job.count * kElemBytes;
@@ -1052,15 +1190,21 @@ enec_encode_kernel(EncodeJob job, int* status) {
     }
 
     // the previous block of this CTA, whose records wait in the other buffer
-    if (pending_block != 0xFFFFFFFFu)
-        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
+    if (pending_block != 0xFFFFFFFFu) {
+        const BlockCtx& px = s_ctx[BATCH ? (iter + 2) % 3 : 0];
+        resolve_block<DT>(BATCH ? px.job : single, BATCH ? px.tensor : single_tensor, pending_block, pending_wide, pending_bad,
+                          s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
+    }
     pending_block = k;
     pending_wide = wide_count;
     pending_bad = any_bad != 0;
     cur ^= 1;
     }
-    if (pending_block != 0xFFFFFFFFu)
-        resolve_block<DT>(job, tensor, pending_block, pending_wide, pending_bad, s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
+    if (pending_block != 0xFFFFFFFFu) {
+        const BlockCtx& px = s_ctx[BATCH ? (iter + 2) % 3 : 0];
+        resolve_block<DT>(BATCH ? px.job : single, BATCH ? px.tensor : single_tensor, pending_block, pending_wide, pending_bad,
+                          s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
+    }
 }
 
 // Stream of an empty tensor: header and a one-entry table.

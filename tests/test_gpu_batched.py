@@ -99,3 +99,94 @@ def test_host_argument_checks():
     assert enec.enec_decompress_batched([(buf[1:], 4000, out, 64)], 0) == -1
     assert enec.enec_decompress_batched([(buf, 10, out, 64)], 0) == -4
     torch.cuda.synchronize()
+
+
+# ---- enec_compress_batched ---------------------------------------------------------------------------
+def _compress_batched(words_list, dt):
+    import paper_2604_03298_b200 as enec
+    from gpu_util import status_tensor
+    dtype = {0: torch.bfloat16, 1: torch.float16, 2: torch.float32}[dt]
+    view = np.int32 if dt == 2 else np.int16
+    srcs = [torch.from_numpy(w.view(view).copy()).cuda().view(dtype) if w.size else torch.empty(0, dtype=dtype, device="cuda")
+            for w in words_list]
+    caps = [enec.enec_max_compressed_size(dt, int(w.size)) for w in words_list]
+    bufs = [torch.full((c + 64,), 0xA5, dtype=torch.uint8, device="cuda") for c in caps]
+    sizes = torch.zeros(len(words_list), dtype=torch.int64, device="cuda")
+    status = status_tensor()
+    items = [(s, b, int(w.size), c) for s, b, w, c in zip(srcs, bufs, words_list, caps)]
+    st = enec.enec_compress_batched(items, dt, sizes, status)
+    torch.cuda.synchronize()
+    for b, c in zip(bufs, caps):
+        assert (b[c:] == 0xA5).all(), "write behind an output buffer"
+    return st, int(status.item()), [b[:n].cpu().numpy() for b, n in zip(bufs, sizes.tolist())]
+
+
+def _gaussian16(count, seed, dtype=torch.bfloat16, sigma=0.02, mean=0.0):
+    g = torch.Generator().manual_seed(seed)
+    return (torch.randn(count, generator=g) * sigma + mean).to(dtype).view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("dt", [0, 1])
+def test_compress_batched_matches_the_oracle_per_tensor(oracle, dt):
+    dtype = torch.bfloat16 if dt == 0 else torch.float16
+    counts = [16384 * 30 + 11, 2048, 16, 0, 16384, 5, 16384 * 7, 2048, 100, 16384 * 64 + 1, 4096, 33]
+    ws = [_gaussian16(c, 900 + i, dtype, sigma=0.02 if i % 3 else 0.5, mean=1.0 if i % 4 == 1 else 0.0) for i, c in enumerate(counts)]
+    st, dev, got = _compress_batched(ws, dt)
+    assert (st, dev) == (0, 0)
+    for i, (w, g) in enumerate(zip(ws, got)):
+        want = oracle.compress(w, dt)
+        assert g.size == want.size and np.array_equal(g, want), f"tensor {i} (count {w.size}): stream differs"
+
+
+def test_compress_batched_fp32(oracle):
+    rng = np.random.default_rng(12)
+    ws = []
+    for i, c in enumerate([16384 * 9 + 3, 64, 16384 * 2, 7, 2048]):
+        g = torch.Generator().manual_seed(40 + i)
+        ws.append((torch.randn(c, generator=g) * 0.02).view(torch.int32).numpy().view(np.uint32))
+    st, dev, got = _compress_batched(ws, 2)
+    assert (st, dev) == (0, 0)
+    for i, (w, g) in enumerate(zip(ws, got)):
+        assert np.array_equal(g, oracle.compress(w, 2)), f"tensor {i}"
+
+
+def test_compress_batched_many_small_tensors_round_trip(oracle):
+    """The shape of the MoE set at reduced size: expert matrices plus hundreds of one-block vectors, compressed by
+    one call and decompressed by one call; a sample is compared with the oracle."""
+    import paper_2604_03298_b200 as enec
+    from gpu_util import status_tensor
+    counts = [176 * 16384 // 8] * 24 + [2048] * 700
+    srcs = [(torch.randn(c, device="cuda", generator=torch.Generator(device="cuda").manual_seed(i)) * 0.02).to(torch.bfloat16)
+            for i, c in enumerate(counts)]
+    caps = [enec.enec_max_compressed_size(0, c) for c in counts]
+    bufs = [torch.empty(c, dtype=torch.uint8, device="cuda") for c in caps]
+    sizes = torch.zeros(len(counts), dtype=torch.int64, device="cuda")
+    status = status_tensor()
+    for _ in range(2):   # twice: the call's scratch area is reused
+        assert enec.enec_compress_batched([(s, b, c, cap) for s, b, c, cap in zip(srcs, bufs, counts, caps)], 0, sizes, status) == 0
+    outs = [torch.zeros_like(s) for s in srcs]
+    nbytes = sizes.tolist()
+    assert enec.enec_decompress_batched([(b, n, o, c) for b, n, o, c in zip(bufs, nbytes, outs, counts)], 0, status) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for s, o in zip(srcs, outs):
+        assert torch.equal(s.view(torch.int16), o.view(torch.int16))
+    for i in (0, 23, 24, 300, 723):
+        want = oracle.compress(s_words(srcs[i]), 0)
+        assert np.array_equal(bufs[i][:nbytes[i]].cpu().numpy(), want)
+
+
+def s_words(t):
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def test_compress_batched_argument_checks():
+    import paper_2604_03298_b200 as enec
+    src = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
+    cap = enec.enec_max_compressed_size(0, 4096)
+    dst = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    assert enec.enec_compress_batched([], 0) == 0
+    assert enec.enec_compress_batched([(src, dst, 4096, cap)], 9) == -2
+    assert enec.enec_compress_batched([(src, dst, 4096, cap - 1)], 0) == -3
+    assert enec.enec_compress_batched([(src[1:], dst, 4000, cap)], 0) == -1
+    torch.cuda.synchronize()
