@@ -28,6 +28,9 @@ WORKLOADS = {
     "layer": (2, "one Llama-3-8B-shaped decoder layer in bf16, 9 tensors, 436 MB"),
     "tensor": (1, "one bf16 tensor 1024x4096, 8 MB"),
     "layer_fp32": (7, "one OLMo-1B-shaped decoder layer in fp32, 7 tensors, 268 MB (side measurement)"),
+    "heavy": (4, "heavy-tailed stress set: 64 fp16 + 64 bf16 tensors 4096x4096 (Laplace / Student-t, outliers, zeros), 4.3 GB"),
+    "moe": (5, "many-small-tensor MoE set: 768 bf16 expert matrices + 4096 vectors of 2048, 4864 tensors, 4.4 GB; "
+               "the step uses the batched entry points"),
     "olmo1b_fp32": (6, "OLMo-1B-shaped fp32 weight set, 115 tensors, 5.1 GB (side measurement: Sec. 6.2 fp32 support)"),
 }
 SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -192,6 +195,7 @@ def run_ours(args):
     enec.lib()  # fails loudly if libenec.so is missing
 
     cfg, desc = WORKLOADS[args.workload]
+    batched_step = cfg == 5   # the set made for enec_compress_batched / enec_decompress_batched
     specs = synth.config_specs(cfg)
     # weak scaling: every rank holds a full copy of the set drawn with its own seeds
     import dataclasses
@@ -207,9 +211,21 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     # warm-up steps, then one verified round trip (outside the timed region)
+    def compress_pass():
+        if batched_step:
+            cs.compress_batched()
+        else:
+            cs.compress_all(n_streams=args.streams)
+
+    def decompress_pass():
+        if batched_step:
+            cs.decompress_batched()
+        else:
+            cs.decompress_all(n_streams=args.streams)
+
     for _ in range(max(args.warmup, 1)):
-        cs.compress_all(n_streams=args.streams)
-        cs.decompress_all(n_streams=args.streams)
+        compress_pass()
+        decompress_pass()
     torch.cuda.synchronize()
     cs.check_status()
     cs.verify_roundtrip()
@@ -228,9 +244,9 @@ def run_ours(args):
     t0 = time.perf_counter()
     for k in range(args.steps):
         ev[k][0].record()
-        cs.compress_all(n_streams=args.streams)
+        compress_pass()
         ev[k][1].record()
-        cs.decompress_all(n_streams=args.streams)
+        decompress_pass()
         ev[k][2].record()
     barrier()
     wall_ms = (time.perf_counter() - t0) * 1e3
@@ -247,7 +263,7 @@ def run_ours(args):
 
     # end to end through host buffers (pinned): host stream -> device -> decompress -> host tensor, and the
     # compress direction likewise, on one decoder layer of this rank's set
-    layer = [i for i, s in enumerate(specs) if s.name.startswith("l0.") or cfg == 1][:9]
+    layer = [i for i, s in enumerate(specs) if s.name.startswith("l0.")][:9] or list(range(min(9, len(specs))))
     h_streams = [torch.empty(int(cs.sizes[i].item()), dtype=torch.uint8).pin_memory() for i in layer]
     h_raw = [torch.empty(cs.raw[i].numel(), dtype=cs.raw[i].dtype).pin_memory() for i in layer]
     for h, i in zip(h_streams, layer):
@@ -297,12 +313,12 @@ def run_ours(args):
     # the same decompress pass as one batched launch (not part of `value`: the workload says tensor by tensor)
     sizes_host = cs.sizes.cpu().tolist()
     one_dtype = len({t.dtype for t in cs.raw}) == 1   # a batched launch takes tensors of one dtype
-    batch_items = [(cs.streams[i], sizes_host[i], cs.outs[i], t.numel()) for i, t in enumerate(cs.raw)]
 
     def batched_pass():
-        assert enec.enec_decompress_batched(batch_items, dtype_code(cs.raw[0].dtype), cs.status) == 0
+        cs.decompress_batched()
 
     ms_batched = time_e2e(batched_pass) if one_dtype else None
+    ms_comp_batched = time_e2e(cs.compress_batched)
     # the same steps again with the calls spread over several streams (the timed step itself keeps the
     # workload's "tensor by tensor on one stream" unless --streams says otherwise)
     for _ in range(2):
@@ -334,7 +350,7 @@ def run_ours(args):
         return
 
     peak, peak_kind = measured_peak_gbs()
-    n_dec = len(cs.raw)
+    n_dec = len({t.dtype for t in cs.raw}) if batched_step else len(cs.raw)   # decode launches of a step
     dec_moved = (raw_bytes + comp_bytes)                       # algorithmic bytes of one decompress pass (this rank)
     achieved = dec_moved / (ms_dec * 1e-3) / 1e9
     elems = sum(t.numel() for t in cs.raw)
@@ -369,8 +385,10 @@ def run_ours(args):
         "metric": METRIC, "value": total_raw / (ms_dec * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": desc, "tensors_per_rank": n_dec, "raw_bytes_per_rank": raw_bytes,
-                   "step": "enec_compress of every tensor, then enec_decompress of every tensor; tensor i on side "
+        "config": {"workload": desc, "tensors_per_rank": len(cs.raw), "raw_bytes_per_rank": raw_bytes,
+                   "step": "enec_compress_batched of the set, then enec_decompress_batched of the set, one stream"
+                           if batched_step else
+                           "enec_compress of every tensor, then enec_decompress of every tensor; tensor i on side "
                            f"stream i mod {args.streams}, forked from and joined to the timed stream with events"
                            if args.streams > 1 else
                            "enec_compress of every tensor, then enec_decompress of every tensor, one stream",
@@ -392,6 +410,9 @@ def run_ours(args):
         "decompress_batched": None if ms_batched is None else {
             "value": total_raw / (ms_batched * 1e-3) / 1e9, "unit": "GB/s", "launches_per_pass": 1,
             "note": "same streams through enec_decompress_batched, one launch for the whole set"},
+        "compress_batched": {"value": total_raw / (ms_comp_batched * 1e-3) / 1e9, "unit": "GB/s",
+                             "launches_per_pass": 2 * len({t.dtype for t in cs.raw}),
+                             "note": "same tensors through enec_compress_batched (one call per dtype of the set)"},
         "compression_ratio": total_raw / total_comp,
         "roofline": roofline,
         "cpu_baseline": cpu,

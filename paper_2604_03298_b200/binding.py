@@ -95,20 +95,26 @@ def enec_decompress(d_in, in_size, dt, count, d_out, d_status=None) -> int:
     return lib().enec_decompress(_ptr(d_in), in_size, dt, count, _ptr(d_out), _ptr(d_status), _stream())
 
 
-def enec_decompress_batched(items, dt, d_status=None) -> int:
-    """items: list of (stream_tensor, stream_bytes, out_tensor, count)."""
+def make_batch(items):
+    """The C array of enec_batch_item for a list of (in_tensor, out_tensor, count, size) tuples. A caller that
+    repeats a batched call on the same buffers can build it once and pass it instead of the list."""
     arr = (BatchItem * len(items))()
-    for i, (src, nbytes, dst, count) in enumerate(items):
-        arr[i].d_in, arr[i].d_out, arr[i].count, arr[i].size = src.data_ptr(), dst.data_ptr(), count, nbytes
-    return lib().enec_decompress_batched(C.cast(arr, C.c_void_p), len(items), dt, _ptr(d_status), _stream())
+    for i, (src, dst, count, size) in enumerate(items):
+        arr[i].d_in, arr[i].d_out, arr[i].count, arr[i].size = src.data_ptr(), dst.data_ptr(), count, size
+    return arr
+
+
+def enec_decompress_batched(items, dt, d_status=None) -> int:
+    """items: list of (stream_tensor, stream_bytes, out_tensor, count), or a make_batch() array."""
+    arr = items if isinstance(items, C.Array) else make_batch([(src, dst, count, nbytes) for src, nbytes, dst, count in items])
+    return lib().enec_decompress_batched(C.cast(arr, C.c_void_p), len(arr), dt, _ptr(d_status), _stream())
 
 
 def enec_compress_batched(items, dt, d_out_sizes=None, d_status=None) -> int:
-    """items: list of (tensor, stream_buffer, count, capacity); d_out_sizes: int64 CUDA tensor [len(items)] or None."""
-    arr = (BatchItem * len(items))()
-    for i, (src, dst, count, capacity) in enumerate(items):
-        arr[i].d_in, arr[i].d_out, arr[i].count, arr[i].size = src.data_ptr(), dst.data_ptr(), count, capacity
-    return lib().enec_compress_batched(C.cast(arr, C.c_void_p), len(items), dt, _ptr(d_out_sizes), _ptr(d_status),
+    """items: list of (tensor, stream_buffer, count, capacity), or a make_batch() array; d_out_sizes: int64 CUDA
+    tensor [len(items)] or None."""
+    arr = items if isinstance(items, C.Array) else make_batch(items)
+    return lib().enec_compress_batched(C.cast(arr, C.c_void_p), len(arr), dt, _ptr(d_out_sizes), _ptr(d_status),
                                        _stream())
 
 

@@ -52,6 +52,7 @@ class CodecSet:
     sizes: Optional[torch.Tensor] = None      # int64 [n]: stream lengths, written by the device
     status: Optional[torch.Tensor] = None     # int32 [1]: first device error of any call
     shared_outs: bool = False
+    batches: Optional[list] = None   # cached item arrays of the batched calls
     side: List[torch.cuda.Stream] = field(default_factory=list)   # side streams of the multi-stream passes
 
     @classmethod
@@ -132,6 +133,42 @@ class CodecSet:
                                   self.outs[i], self.status)
         if st != 0:
             raise enec.EnecError(st, f"enec_decompress tensor {i}")
+
+    def _dtype_groups(self):
+        groups = {}
+        for i, t in enumerate(self.raw):
+            groups.setdefault(t.dtype, []).append(i)
+        return groups
+
+    def _batches(self):
+        """Per dtype of the set: the item arrays of the two batched calls, built once (the buffers do not move)."""
+        if self.batches is None:
+            self.batches = []
+            for dtype, idx in self._dtype_groups().items():
+                whole = len(idx) == len(self.raw)
+                comp = enec.make_batch([(self.raw[i], self.streams[i], self.raw[i].numel(), self.streams[i].numel()) for i in idx])
+                dec = enec.make_batch([(self.streams[i], self.outs[i], self.raw[i].numel(), self.streams[i].numel()) for i in idx])
+                sizes = self.sizes if whole else torch.zeros(len(idx), dtype=torch.int64, device=self.sizes.device)
+                where = None if whole else torch.tensor(idx, device=self.sizes.device)
+                self.batches.append((_DT[dtype], comp, dec, sizes, where))
+        return self.batches
+
+    def compress_batched(self) -> None:
+        """One enec_compress_batched call per dtype of the set (two launches each) on the current stream."""
+        for dt, comp, _, sizes, where in self._batches():
+            st = enec.enec_compress_batched(comp, dt, sizes, self.status)
+            if st != 0:
+                raise enec.EnecError(st, "enec_compress_batched")
+            if where is not None:
+                self.sizes[where] = sizes
+
+    def decompress_batched(self) -> None:
+        """One enec_decompress_batched call (one launch) per dtype of the set on the current stream. The stream
+        length passed is the buffer's capacity, as in decompress_all."""
+        for dt, _, dec, _, _ in self._batches():
+            st = enec.enec_decompress_batched(dec, dt, self.status)
+            if st != 0:
+                raise enec.EnecError(st, "enec_decompress_batched")
 
     def check_status(self) -> None:
         code = int(self.status.item())

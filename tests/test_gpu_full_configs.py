@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 SPREAD_STREAMS = 8   # bench.py's --spread-streams default
 
 
-def _run_set(specs, oracle, sample, reuse=None, n_streams=1):
+def _run_set(specs, oracle, sample, reuse=None, n_streams=1, batched=False):
     import paper_2604_03298_b200 as enec
     from paper_2604_03298_b200 import runner, synth
     cache = {}
@@ -26,8 +26,12 @@ def _run_set(specs, oracle, sample, reuse=None, n_streams=1):
             cache[key] = synth.make_tensor(s, "cuda")
         raw.append(cache[key])
     cs = runner.CodecSet.allocate(raw)
-    cs.compress_all(n_streams=n_streams)
-    cs.decompress_all(n_streams=n_streams)
+    if batched:
+        cs.compress_batched()
+        cs.decompress_batched()
+    else:
+        cs.compress_all(n_streams=n_streams)
+        cs.decompress_all(n_streams=n_streams)
     torch.cuda.synchronize()
     cs.check_status()
     cs.verify_roundtrip()
@@ -72,21 +76,24 @@ def test_config3_llama8b_full(oracle, n_streams):
     assert 1.36 < ratio < 1.40                                          # Table 4 reports 1.36 for Llama-3.1-8B
 
 
-def test_config4_heavy_tailed_full(oracle):
+@pytest.mark.parametrize("batched", [False, True])
+def test_config4_heavy_tailed_full(oracle, batched):
     from paper_2604_03298_b200 import synth
     specs = synth.config_specs(4)
     assert len(specs) == 128 and specs[0].shape == (4096, 4096)
-    ratio = _run_set(specs, oracle, sample=(0, 31, 45, 63, 64, 95, 100, 127))
+    ratio = _run_set(specs, oracle, sample=(0, 31, 45, 63, 64, 95, 100, 127), batched=batched)
     assert 1.0 < ratio < 1.35                                           # zeros force the full exponent width
 
 
-def test_config5_moe_full(oracle):
+@pytest.mark.parametrize("batched", [True, False])
+def test_config5_moe_full(oracle, batched):
+    """Through the batched entry points (the way this set is meant to be run) and tensor by tensor."""
     from paper_2604_03298_b200 import synth
     specs = synth.config_specs(5)
     assert len(specs) == 768 + 4096
     # expert matrices share three shapes and one distribution: 24 distinct draws stand for the 768
     reuse = lambda i, s: (s.shape, i % 24) if len(s.shape) == 2 else ("v", i)
-    ratio = _run_set(specs, oracle, sample=(0, 1, 2, 767, 768, 769, 2000, 4863), reuse=reuse)
+    ratio = _run_set(specs, oracle, sample=(0, 1, 2, 767, 768, 769, 2000, 4863), reuse=reuse, batched=batched)
     assert 1.36 < ratio < 1.40
 
 
