@@ -433,10 +433,10 @@ def run_ours(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per element of enec_decode_kernel from the committed ncu capture
-# (profiles/decode_kernel_llama_layer.md: 85.54 MB read + 61.83 MB written for the 58,720,256 elements of
+# (profiles/decode_kernel_llama_layer.md: 85.54 MB read + 62.36 MB written for the 58,720,256 elements of
 # gate_proj). Below the algorithmic 3.475 B/element because part of the output is still dirty in L2 when the
 # kernel ends. Set to None when the kernel changes until a new capture exists.
-DECODE_DRAM_BYTES_PER_ELEM = (85.538048e6 + 61.829120e6) / 58720256
+DECODE_DRAM_BYTES_PER_ELEM = (85.537024e6 + 62.355456e6) / 58720256
 
 
 def main():
