@@ -144,7 +144,7 @@ enec_status enec_compress_batched(const enec_batch_item* h_items, int n_items, e
  *     that first call outside any stream capture.
  */
 #define ENEC_NOALLOC_MAX_COUNT ((size_t)1 << 30)
-#define ENEC_NOALLOC_SCRATCH_BYTES (4096 + (ENEC_NOALLOC_MAX_COUNT / 16384) * 8)
+#define ENEC_NOALLOC_SCRATCH_BYTES (8192 + (ENEC_NOALLOC_MAX_COUNT / 16384) * 8)
 enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
                                   size_t* d_out_size, int* d_status, enec_stream_t stream);
 

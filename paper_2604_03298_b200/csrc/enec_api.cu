@@ -255,6 +255,7 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
 constexpr uint64_t kNoAllocMaxCount = uint64_t(1) << 30;
 constexpr size_t kNoAllocScratchBytes = kControlBytes + size_t(kNoAllocMaxCount / kBlockElems) * sizeof(unsigned long long);
 static __device__ __align__(256) uint8_t g_noalloc_scratch[kNoAllocScratchBytes];
+static_assert(kNoAllocScratchBytes == ENEC_NOALLOC_SCRATCH_BYTES, "the header states the size of the built-in scratch");
 
 // Device address of the scratch on the current device, looked up once per device.
 static enec_status noalloc_scratch(int dev, uint8_t** out) {
