@@ -74,7 +74,7 @@ enec_status enec_compress(const void* d_in, enec_dtype dt, size_t count, void* d
 
 /*
  * As enec_compress, with the caller's (b, n, m) instead of the search of Sec. 5.5 (the paper's offline
- * tuned mode, Sec. 6.1 "Compression Configurations"). 0 <= b < 2^E, 1 <= m <= n <= E (E = 8 for bf16,
+ * tuned mode, Sec. 6 "Compression Configurations"). 0 <= b < 2^E, 1 <= m <= n <= E (E = 8 for bf16,
  * 5 for fp16). If some exponent of the tensor does not survive (b, n) the device reports
  * ENEC_ERR_PARAMS_NOT_LOSSLESS in *d_status and writes no stream.
  */

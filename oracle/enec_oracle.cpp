@@ -12,6 +12,7 @@
 #include "enec_oracle.h"
 
 #include <cstring>
+#include <algorithm>
 #include <vector>
 
 namespace {
@@ -72,13 +73,15 @@ Geometry geometry(size_t count) {
 }
 
 struct Sections {
-    size_t table, mask, low, smhi, sm, smlo, high, total;
+    size_t unmap, table, mask, low, smhi, sm, smlo, high, total;
 };
 
-// Section offsets for stored widths (n, m) and a_total anomalous groups.
-Sections sections(int dtype, size_t count, const Geometry& g, int n, int m, uint64_t a_total) {
+// Section offsets for stored widths (n, m) and a_total anomalous groups. Streams of the frequency-rank variant
+// carry a 256-byte table (rank -> exponent) between the header and the prefix table.
+Sections sections(int dtype, size_t count, const Geometry& g, int n, int m, uint64_t a_total, bool ranked = false) {
     Sections s;
-    s.table = kHeaderBytes;
+    s.unmap = kHeaderBytes;
+    s.table = kHeaderBytes + (ranked ? 256 : 0);
     s.mask = s.table + align16(4 * (size_t(g.nblocks) + 1));
     s.low = s.mask + align16((size_t(g.total_groups) + 7) / 8);
     s.smhi = s.low + align16(size_t(g.padded_count) * m / 8);
@@ -251,6 +254,38 @@ void param_search(const uint64_t* hist, int E, int* b_out, int* n_out, int* m_ou
     *b_out = best_b; *n_out = best_n; *m_out = best_m;
 }
 
+// ---- the frequency-rank variant (Sec. 4.2, Algorithm 1: E' = T_freq[E], "the sorted frequency indices serve as
+// mapping values"; the ablation's V1 keeps that mapping and adds the one-bit group mask and Algorithm 2) ----
+// rank_of[x] = position of exponent x when the occupied exponents are sorted by falling count (ties: smaller
+// exponent first); unmap[r] = the exponent of rank r. The stored value of an element is its rank: no base, no
+// sign bit, n = bits needed for the largest rank, m by Eq. 4 over the ranks' bit widths.
+void rank_mapping(const uint64_t* hist, int E, uint8_t* rank_of, uint8_t* unmap, int* n_out, int* m_out) {
+    const int bins = 1 << E;
+    std::vector<int> order;
+    uint64_t total = 0;
+    for (int x = 0; x < bins; ++x) if (hist[x]) { order.push_back(x); total += hist[x]; }
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return hist[a] > hist[b]; });
+    std::memset(rank_of, 0, 256);
+    std::memset(unmap, 0, 256);
+    for (size_t r = 0; r < order.size(); ++r) { rank_of[order[r]] = uint8_t(r); unmap[r] = uint8_t(order[r]); }
+    int n = order.size() <= 1 ? 1 : bit_width(uint64_t(order.size() - 1));
+    int best_m = 1;
+    double best_bexp = 0.0;
+    for (int m = 1; m <= n; ++m) {
+        uint64_t cnt = 0;
+        for (size_t r = 0; r < order.size(); ++r) if (bit_width(uint64_t(r)) <= m) cnt += hist[order[r]];
+        double p = total ? double(cnt) / double(total) : 1.0;
+        double p2 = p * p;
+        double p4 = p2 * p2;
+        double p8 = p4 * p4;
+        double p16 = p8 * p8;
+        double saving = double(m - n) * p16;
+        double bexp = (double(n) + 0.0625) + saving;
+        if (m == 1 || bexp < best_bexp) { best_m = m; best_bexp = bexp; }
+    }
+    *n_out = n; *m_out = best_m;
+}
+
 // Whether (b, n) reproduces every exponent in [l, h] (n == E always does).
 bool params_lossless(int b, int n, int l, int h, int E) {
     if (n == E) return true;
@@ -279,7 +314,7 @@ uint32_t load_word(const void* in, int dtype, size_t i) {
 }
 
 int encode(const void* in, int dtype, size_t count, bool have_params, int b, int n, int m,
-           uint8_t* out, size_t capacity, size_t* out_size) {
+           uint8_t* out, size_t capacity, size_t* out_size, bool ranked = false) {
     if (!known_dtype(dtype)) return ERR_UNSUPPORTED_DTYPE;
     if ((!in && count) || !out || !out_size || (count >> 36)) return ERR_INVALID_ARG;
     const int E = exp_bits(dtype);
@@ -295,7 +330,12 @@ int encode(const void* in, int dtype, size_t count, bool have_params, int b, int
         x[i] = uint8_t(xe); sm[i] = s;
         hist[xe] += 1;
     }
-    if (!have_params) {
+    uint8_t rank_of[256], unmap[256];
+    if (ranked) {
+        if (have_params) return ERR_INVALID_ARG;
+        rank_mapping(hist.data(), E, rank_of, unmap, &n, &m);
+        b = 0;
+    } else if (!have_params) {
         param_search(hist.data(), E, &b, &n, &m, nullptr, nullptr);
     } else {
         if (n < 1 || n > E || m < 1 || m > n || b < 0 || b >= (1 << E)) return ERR_INVALID_ARG;
@@ -316,7 +356,7 @@ int encode(const void* in, int dtype, size_t count, bool have_params, int b, int
         uint32_t np = (k + 1 == g.nblocks) ? g.tail_padded : kBlock;
         std::vector<uint16_t> y(np, 0), hi3(np, 0);  // padding: y = 0
         for (uint32_t i = 0; i < real; ++i) {
-            y[i] = uint16_t(transform(x[first + i], b, n));
+            y[i] = ranked ? uint16_t(rank_of[x[first + i]]) : uint16_t(transform(x[first + i], b, n));
             if (dtype == 1) hi3[i] = uint16_t(sm[first + i] >> 8);  // sign | mant[9:8]
         }
         table[k] = a_total;
@@ -344,13 +384,15 @@ int encode(const void* in, int dtype, size_t count, bool have_params, int b, int
     }
     table[g.nblocks] = a_total;
 
-    const Sections s = sections(dtype, count, g, n, m, a_total);
+    const Sections s = sections(dtype, count, g, n, m, a_total, ranked);
     *out_size = s.total;
     if (capacity < s.total) return ERR_BUFFER_TOO_SMALL;
     std::memset(out, 0, s.total);
     std::memcpy(out, "ENEC", 4);
     put_u16(out + 4, 1);
     out[6] = uint8_t(dtype);
+    out[7] = ranked ? 1 : 0;  // variant: 0 = linear transform, 1 = frequency ranks
+    if (ranked) std::memcpy(out + s.unmap, unmap, 256);
     put_u64(out + 8, count);
     put_u32(out + 16, kBlock);
     out[20] = uint8_t(b); out[21] = uint8_t(n); out[22] = uint8_t(m); out[23] = uint8_t(kGroup);
@@ -384,11 +426,12 @@ int decode(const uint8_t* in, size_t in_size, int dtype, size_t count, void* out
         return ERR_BAD_STREAM;
     const int E = exp_bits(dtype);
     const int b = in[20], n = in[21], m = in[22];
-    if (n < 1 || n > E || m < 1 || m > n || b >= (1 << E)) return ERR_BAD_STREAM;
+    if (n < 1 || n > E || m < 1 || m > n || b >= (1 << E) || in[7] > 1) return ERR_BAD_STREAM;
+    const bool ranked = in[7] == 1;
     const Geometry g = geometry(count);
     const uint32_t a_total = get_u32(in + 32);
     if (get_u32(in + 24) != g.nblocks || get_u32(in + 28) != g.total_groups) return ERR_BAD_STREAM;
-    const Sections s = sections(dtype, count, g, n, m, a_total);
+    const Sections s = sections(dtype, count, g, n, m, a_total, ranked);
     if (get_u64(in + 40) != s.total || in_size < s.total) return ERR_BAD_STREAM;
     if (get_u32(in + s.table + 4 * size_t(g.nblocks)) != a_total) return ERR_BAD_STREAM;
 
@@ -414,7 +457,7 @@ int decode(const uint8_t* in, size_t in_size, int dtype, size_t count, void* out
         }
         if (rank != next) return ERR_BAD_STREAM;  // table must agree with the mask's popcount
         for (uint32_t i = 0; i < real; ++i) {
-            uint32_t xe = inverse_transform(y[i], b, n, E);
+            uint32_t xe = ranked ? in[s.unmap + (y[i] & 0xFF)] : inverse_transform(y[i], b, n, E);
             uint32_t smv = in[s.sm + first + i];
             if (dtype == 1) smv |= uint32_t(hi3[i]) << 8;
             if (dtype == 2) {
@@ -475,6 +518,16 @@ int enec_oracle_compress_with_params(const void* in, int dtype, size_t count, in
                                      size_t capacity, size_t* out_size) {
     return encode(in, dtype, count, true, b, n, m,
                   static_cast<uint8_t*>(out), capacity, out_size);
+}
+
+// The frequency-rank variant stores its 256-byte table on top of the same sections.
+size_t enec_oracle_max_compressed_size_ranked(int dtype, size_t count) {
+    const size_t base = enec_oracle_max_compressed_size(dtype, count);
+    return base ? base + 256 : 0;
+}
+
+int enec_oracle_compress_ranked(const void* in, int dtype, size_t count, void* out, size_t capacity, size_t* out_size) {
+    return encode(in, dtype, count, false, 0, 0, 0, static_cast<uint8_t*>(out), capacity, out_size, true);
 }
 
 int enec_oracle_decompress(const void* in, size_t in_size, int dtype, size_t count, void* out) {

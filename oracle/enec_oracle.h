@@ -44,6 +44,11 @@ void enec_oracle_alg2_unpack(const uint8_t* in, size_t N, int a, uint16_t* out);
 
 /* Whole codec over host memory. */
 size_t enec_oracle_max_compressed_size(int dtype, size_t count);
+/* The frequency-rank variant (Sec. 4.2, Algorithm 1; the ablation's V1): stored value = rank of the exponent by
+ * falling frequency; header byte 7 = 1; a 256-byte rank -> exponent table follows the header. */
+size_t enec_oracle_max_compressed_size_ranked(int dtype, size_t count);
+int enec_oracle_compress_ranked(const void* in, int dtype, size_t count, void* out, size_t capacity, size_t* out_size);
+
 int enec_oracle_compress(const void* in, int dtype, size_t count, void* out, size_t capacity,
                          size_t* out_size);
 int enec_oracle_compress_with_params(const void* in, int dtype, size_t count, int b, int n, int m,

@@ -42,6 +42,11 @@ def lib():
         L.enec_oracle_alg2_unpack.restype = None
         L.enec_oracle_max_compressed_size.argtypes = [C.c_int, C.c_size_t]
         L.enec_oracle_max_compressed_size.restype = C.c_size_t
+        L.enec_oracle_max_compressed_size_ranked.argtypes = [C.c_int, C.c_size_t]
+        L.enec_oracle_max_compressed_size_ranked.restype = C.c_size_t
+        L.enec_oracle_compress_ranked.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_void_p, C.c_size_t,
+                                                  C.POINTER(C.c_size_t)]
+        L.enec_oracle_compress_ranked.restype = C.c_int
         L.enec_oracle_compress.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_void_p, C.c_size_t,
                                            C.POINTER(C.c_size_t)]
         L.enec_oracle_compress.restype = C.c_int
@@ -125,6 +130,18 @@ def compress(words, dtype, params=None):
         b, n, m = params
         st = lib().enec_oracle_compress_with_params(words.ctypes.data, dtype, words.size, b, n, m,
                                                     out.ctypes.data, cap, C.byref(size))
+    if st != 0:
+        raise OracleError(st)
+    return out[:size.value].copy()
+
+
+def compress_ranked(words, dtype):
+    """The frequency-rank variant of compress(): same stream sections plus the rank -> exponent table."""
+    words = np.ascontiguousarray(words, dtype=np.uint32 if dtype == FP32 else np.uint16).reshape(-1)
+    cap = lib().enec_oracle_max_compressed_size_ranked(dtype, words.size)
+    out = np.empty(cap, dtype=np.uint8)
+    size = C.c_size_t(0)
+    st = lib().enec_oracle_compress_ranked(words.ctypes.data, dtype, words.size, out.ctypes.data, cap, C.byref(size))
     if st != 0:
         raise OracleError(st)
     return out[:size.value].copy()

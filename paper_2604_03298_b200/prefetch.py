@@ -1,5 +1,5 @@
-"""Layer-wise weight prefetch: decompress layer i + 1 on a side stream while layer i computes (Sec. 6.1
-"End-to-end inference": the paper overlaps layer-wise decompression with the forward pass).
+"""Layer-wise weight prefetch: decompress layer i + 1 on a side stream while layer i computes (Sec. 6.3
+"End-to-End Inference Speedup": the paper overlaps layer-wise decompression with the forward pass).
 
 The weights of all layers stay compressed in device memory; two layer-sized buffers hold the layer being used
 and the layer being decompressed. Each layer is one `enec_decompress_batched` launch on the side stream; CUDA

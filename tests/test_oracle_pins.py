@@ -473,3 +473,75 @@ def test_fp32_gaussian_lands_on_table5_and_table4(oracle):
     s = oracle.compress(w, 2)
     assert 119 <= int(s[20]) <= 125 and (int(s[21]), int(s[22])) == (6, 3)
     assert 1.13 < w.nbytes / s.size < 1.18
+
+
+# ---------------------------------------------------------------- frequency-rank variant (Sec. 4.2, Algorithm 1)
+def test_ranked_stream_hand(oracle):
+    fx = read_fixture("stream_hand_ranked.txt")
+    words = np.array([int(t, 16) for t in fx["words"][0].split()], dtype=np.uint16)
+    unmap = np.zeros(256, np.uint8)
+    head = hexbytes(fx["unmap_head"][0])
+    unmap[:head.size] = head
+    expect = np.concatenate([hexbytes(fx["header"][0]), unmap] + [hexbytes(fx[k][0]) for k in ("table", "mask", "low", "sm", "high")])
+    got = oracle.compress_ranked(words, 0)
+    assert got.tolist() == expect.tolist()
+    assert oracle.decompress(got, 0, words.size).tolist() == words.tolist()
+
+
+def test_ranked_table_sorts_exponents_by_falling_count(oracle):
+    rng = np.random.default_rng(4)
+    x = rng.choice(np.arange(100, 140), size=50000, p=np.r_[np.full(20, 0.04), np.full(20, 0.01)]).astype(np.uint16)
+    x[:7] = 3                       # a rare exponent far away, and ties among the plentiful ones are likely
+    words = (x << 7) | rng.integers(0, 128, x.size).astype(np.uint16)
+    s = oracle.compress_ranked(words, 0)
+    counts = np.bincount(x, minlength=256)
+    occupied = int((counts > 0).sum())
+    table = s[64:64 + 256]
+    order = sorted(np.flatnonzero(counts), key=lambda e: (-counts[e], e))     # textbook: count down, exponent up
+    assert table[:occupied].tolist() == order and not table[occupied:].any()
+    n, m = int(s[21]), int(s[22])
+    assert n == max(1, int(occupied - 1).bit_length()) and 1 <= m <= n and s[7] == 1 and s[20] == 0
+    assert np.array_equal(oracle.decompress(s, 0, words.size), words)
+
+
+def test_ranked_cost_never_exceeds_the_linear_transform(oracle):
+    """Sorting by frequency minimises sum count * code over all one-to-one codes (rearrangement inequality), so
+    the rank code's Eq. 3 cost is at most the best linear transform's, for any histogram."""
+    rng = np.random.default_rng(8)
+    for trial in range(40):
+        hist = np.zeros(256, np.uint64)
+        lo = int(rng.integers(0, 200)); width = int(rng.integers(1, 50))
+        hist[lo:lo + width] = rng.integers(0, 10000, width).astype(np.uint64)
+        if not hist.any():
+            continue
+        ranked_cost = int(sum(int(c) * r for r, c in enumerate(sorted((int(v) for v in hist if v), reverse=True))))
+        b, n, m, cost, _ = oracle.param_search(hist, 8)
+        assert ranked_cost <= int(cost[b]), trial
+
+
+def test_ranked_roundtrip_patterns_tails_and_dtypes(oracle):
+    import torch
+    rng = np.random.default_rng(15)
+    for dt in (0, 1):
+        w = rng.permutation(1 << 16).astype(np.uint16)               # every bit pattern: all exponents occupied
+        s = oracle.compress_ranked(w, dt)
+        assert int(s[21]) == (8 if dt == 0 else 5)
+        assert np.array_equal(oracle.decompress(s, dt, w.size), w)
+    for count in (0, 1, 15, 16, 17, 100, 16384, 16385, 16384 * 3 + 5000):
+        g = torch.Generator().manual_seed(count)
+        w = (torch.randn(count, generator=g) * 0.02).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        s = oracle.compress_ranked(w, 0)
+        assert np.array_equal(oracle.decompress(s, 0, count), w)
+    f = (torch.randn(40000, generator=torch.Generator().manual_seed(2)) * 0.02).view(torch.int32).numpy().view(np.uint32)
+    assert np.array_equal(oracle.decompress(oracle.compress_ranked(f, 2), 2, f.size), f)
+    one = np.full(16384 + 3, 0x3F80, np.uint16)                      # one exponent: n = m = 1, every y = 0
+    s = oracle.compress_ranked(one, 0)
+    assert (int(s[21]), int(s[22]), int(s[32])) == (1, 1, 0) and s[64] == 127
+
+
+def test_ranked_is_a_little_smaller_on_gaussian_weights(oracle):
+    """Sec. 6.6 (ablation): the linear transform approximates the frequency order and gives up a little ratio."""
+    import torch
+    w = (torch.randn(1 << 20, generator=torch.Generator().manual_seed(5)) * 0.02).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    linear, ranked = oracle.compress(w, 0).size, oracle.compress_ranked(w, 0).size
+    assert ranked < linear < ranked * 1.03
