@@ -389,6 +389,28 @@ def run_ours(args):
     barrier()
     ms_comp_ms = runner.max_over_ranks(sum(e[0].elapsed_time(e[1]) for e in ev2) / args.steps)
     ms_dec_ms = runner.max_over_ranks(sum(e[1].elapsed_time(e[2]) for e in ev2) / args.steps)
+
+    # ablation: the frequency-rank variant (table look-ups instead of the linear transform), same steps, one stream
+    for _ in range(2):
+        cs.compress_all(ranked=True)
+        cs.decompress_all()
+    torch.cuda.synchronize()
+    cs.check_status()
+    cs.verify_roundtrip()
+    ranked_bytes = runner.sum_over_ranks(cs.compressed_bytes())
+    ev3 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    for k in range(args.steps):
+        ev3[k][0].record()
+        cs.compress_all(ranked=True)
+        ev3[k][1].record()
+        cs.decompress_all()
+        ev3[k][2].record()
+    barrier()
+    ms_comp_ranked = runner.max_over_ranks(sum(e[0].elapsed_time(e[1]) for e in ev3) / args.steps)
+    ms_dec_ranked = runner.max_over_ranks(sum(e[1].elapsed_time(e[2]) for e in ev3) / args.steps)
+    cs.compress_all()      # back to the linear streams for what follows
+    torch.cuda.synchronize()
     cs.check_status()
     cs.verify_roundtrip()
 
@@ -479,6 +501,12 @@ def run_ours(args):
                              "launches_per_pass": 2 * len({t.dtype for t in cs.raw}),
                              "note": "same tensors through enec_compress_batched (one call per dtype of the set)"},
         "compression_ratio": total_raw / total_comp,
+        "ablation_frequency_ranks": {
+            "compression_ratio": total_raw / ranked_bytes,
+            "decompress": {"value": total_raw / (ms_dec_ranked * 1e-3) / 1e9, "unit": "GB/s"},
+            "compress": {"value": total_raw / (ms_comp_ranked * 1e-3) / 1e9, "unit": "GB/s"},
+            "note": "enec_compress_ranked / enec_decompress tensor by tensor on one stream: stored value = rank of the "
+                    "exponent by falling count, looked up in a table (Sec. 4.2, Algorithm 1; the ablation's V1)"},
         "roofline": roofline,
         "cpu_baseline": cpu,
         "cpu_vectorised": cpu_vec,

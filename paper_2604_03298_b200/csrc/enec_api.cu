@@ -144,8 +144,10 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
     if (search) {
         const uint32_t smem = HistShape<DT>::kWarpBytes * (kHistThreads / 32);
         if (!info.hist_attr_set[DT]) {
-            if (cudaFuncSetAttribute(enec_histogram_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) !=
-                cudaSuccess)
+            if (cudaFuncSetAttribute(enec_histogram_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     int(smem)) != cudaSuccess ||
+                cudaFuncSetAttribute(enec_histogram_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     int(smem)) != cudaSuccess)
                 return ENEC_ERR_CUDA;
             info.hist_attr_set[DT] = true;
         }
@@ -153,21 +155,29 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
         uint64_t grid = (chunks + kHistThreads - 1) / kHistThreads;
         if (grid > uint64_t(info.sms) * 3) grid = uint64_t(info.sms) * 3;
         if (grid == 0) grid = 1;
-        if (launch_pdl(enec_histogram_kernel<DT>, uint32_t(grid), kHistThreads, smem, stream, job.in, job.count,
-                       job.ctl) != cudaSuccess)
-            return ENEC_ERR_CUDA;
+        const cudaError_t herr =
+            job.ranked ? launch_pdl(enec_histogram_kernel<DT, true>, uint32_t(grid), kHistThreads, smem, stream, job.in,
+                                    job.count, job.ctl)
+                       : launch_pdl(enec_histogram_kernel<DT, false>, uint32_t(grid), kHistThreads, smem, stream, job.in,
+                                    job.count, job.ctl);
+        if (herr != cudaSuccess) return ENEC_ERR_CUDA;
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
     if (!info.encode_attr_set[DT]) {
-        if (cudaFuncSetAttribute(enec_encode_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(enec_encode_kernel<DT, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(EncodeSmem<DT>::kBytes)) != cudaSuccess ||
+            cudaFuncSetAttribute(enec_encode_kernel<DT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(EncodeSmem<DT>::kBytes)) != cudaSuccess)
             return ENEC_ERR_CUDA;
         info.encode_attr_set[DT] = true;
     }
     uint32_t grid = uint32_t(info.sms) * 4;  // four resident CTAs per SM, each takes block after block
     if (grid > nblocks) grid = nblocks;
-    const cudaError_t err = launch_pdl(enec_encode_kernel<DT, false>, grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream,
-                                       job, EncodeBatch{}, d_status);
+    const cudaError_t err =
+        job.ranked ? launch_pdl(enec_encode_kernel<DT, false, true>, grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream,
+                                job, EncodeBatch{}, d_status)
+                   : launch_pdl(enec_encode_kernel<DT, false, false>, grid, kEncodeThreads, EncodeSmem<DT>::kBytes, stream,
+                                job, EncodeBatch{}, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
@@ -202,19 +212,20 @@ static enec_status launch_encode_batched(const EncodeJob* d_jobs, const HistUnit
 
 static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count, bool with_params, int b, int n,
                                    int m, void* d_out, size_t out_capacity, size_t* d_out_size, int* d_status,
-                                   cudaStream_t stream) {
+                                   cudaStream_t stream, bool ranked = false) {
     if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if ((!d_in && count) || !d_out || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out) ||
         (reinterpret_cast<uintptr_t>(d_out_size) & 7))
         return ENEC_ERR_INVALID_ARG;
     const int E = exp_bits(dt);
     if (with_params && (n < 1 || n > E || m < 1 || m > n || b < 0 || b >= (1 << E))) return ENEC_ERR_INVALID_ARG;
-    if (out_capacity < enec_max_compressed_size(dt, count)) return ENEC_ERR_BUFFER_TOO_SMALL;
+    if (out_capacity < (ranked ? enec_max_compressed_size_ranked(dt, count) : enec_max_compressed_size(dt, count)))
+        return ENEC_ERR_BUFFER_TOO_SMALL;
     unsigned long long* out_size = reinterpret_cast<unsigned long long*>(d_out_size);
     if (count == 0) {
         // no exponent occurs: the search of Sec. 5.5 has nothing to minimise and keeps (0, 1, 1)
         enec_encode_empty_kernel<<<1, 32, 0, stream>>>(static_cast<uint8_t*>(d_out), int(dt), with_params ? b : 0,
-                                                      with_params ? n : 1, with_params ? m : 1, out_size);
+                                                      with_params ? n : 1, with_params ? m : 1, out_size, ranked ? 1 : 0);
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
     }
@@ -240,6 +251,7 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
     job.b = b; job.n = n; job.m = m;
     job.from_search = with_params ? 0 : 1;
     job.check = with_params ? 1 : 0;
+    job.ranked = ranked ? 1 : 0;
     st = dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream)
          : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream)
                            : launch_encode<ENEC_FP32>(job, g.nblocks, !with_params, d_status, info, stream);
@@ -374,6 +386,16 @@ enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t co
 }
 
 
+size_t enec_max_compressed_size_ranked(enec_dtype dt, size_t count) {
+    const size_t base = enec_max_compressed_size(dt, count);
+    return base ? base + kRankTableBytes : 0;
+}
+
+enec_status enec_compress_ranked(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                                 size_t* d_out_size, int* d_status, enec_stream_t stream) {
+    return compress_common(d_in, dt, count, false, 0, 0, 0, d_out, out_capacity, d_out_size, d_status, stream, true);
+}
+
 enec_status enec_compress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, size_t* d_out_sizes,
                                   int* d_status, enec_stream_t stream) {
     if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
@@ -431,6 +453,7 @@ enec_status enec_compress_batched(const enec_batch_item* h_items, int n_items, e
         job.b = 0; job.n = 0; job.m = 0;
         job.from_search = 1;
         job.check = 0;
+        job.ranked = 0;
     }
     memcpy(host.data() + (off_prefix - off_jobs), prefix.data(), prefix.size() * sizeof(uint32_t));
     if (!units.empty()) memcpy(host.data() + (off_units - off_jobs), units.data(), units.size() * sizeof(HistUnit));
@@ -492,6 +515,7 @@ enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count,
     job.b = 0; job.n = 0; job.m = 0;
     job.from_search = 1;
     job.check = 0;
+    job.ranked = 0;
     return dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, true, d_status, info, stream)
            : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, true, d_status, info, stream)
                              : launch_encode<ENEC_FP32>(job, g.nblocks, true, d_status, info, stream);

@@ -21,7 +21,7 @@ struct alignas(16) Header {
     uint32_t magic;         //  0
     uint16_t version;       //  4
     uint8_t dtype;          //  6
-    uint8_t pad0;           //  7
+    uint8_t variant;        //  7: 0 = linear transform (Sec. 5.3), 1 = frequency ranks (Sec. 4.2, Algorithm 1)
     uint64_t count;         //  8
     uint32_t block;         // 16
     uint8_t b, n, m, L;     // 20..23
@@ -60,14 +60,17 @@ __host__ __device__ inline Geometry make_geometry(uint64_t count) {
     return g;
 }
 
+constexpr uint32_t kRankTableBytes = 256;  // frequency-rank variant: rank -> exponent, behind the header
+
 struct Sections {
-    uint64_t table, mask, low, smhi, sm, smlo, high, total;
+    uint64_t unmap, table, mask, low, smhi, sm, smlo, high, total;
 };
 
 __host__ __device__ inline Sections make_sections(int dt, uint64_t count, const Geometry& g, int n, int m,
-                                                  uint64_t a_total) {
+                                                  uint64_t a_total, bool ranked = false) {
     Sections s;
-    s.table = kHeaderBytes;
+    s.unmap = kHeaderBytes;
+    s.table = kHeaderBytes + (ranked ? kRankTableBytes : 0);
     s.mask = s.table + align16(4 * (uint64_t(g.nblocks) + 1));
     s.low = s.mask + align16((uint64_t(g.total_groups) + 7) / 8);
     s.smhi = s.low + align16(g.padded_count * uint64_t(m) / 8);

@@ -177,6 +177,7 @@ struct JobCtx {
     uint32_t nblocks, tail_real, tail_padded;
     uint32_t a_total;
     int b, n, m;
+    bool mapped;  // frequency-rank variant: the stored value is a rank, looked up in the stream's table (behind the header)
     uint64_t off_table, off_mask, off_low, off_smhi, off_sm, off_smlo, off_high, total;
 };
 
@@ -189,12 +190,13 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
         h.block != kBlockElems || h.L != kGroupElems)
         return ENEC_ERR_BAD_STREAM;
     constexpr int E = exp_bits(DT);
-    if (h.n < 1 || h.n > E || h.m < 1 || h.m > h.n || h.b >= (1 << E)) return ENEC_ERR_BAD_STREAM;
+    if (h.n < 1 || h.n > E || h.m < 1 || h.m > h.n || h.b >= (1 << E) || h.variant > 1) return ENEC_ERR_BAD_STREAM;
     const Geometry g = make_geometry(job.count);
     if (h.nblocks != g.nblocks || h.total_groups != g.total_groups || h.a_total > g.total_groups)
         return ENEC_ERR_BAD_STREAM;
-    const Sections s = make_sections(DT, job.count, g, h.n, h.m, h.a_total);
+    const Sections s = make_sections(DT, job.count, g, h.n, h.m, h.a_total, h.variant == 1);
     if (h.total_bytes != s.total || job.in_size < s.total) return ENEC_ERR_BAD_STREAM;
+    c.mapped = h.variant == 1;
     c.in = job.in;
     c.out = job.out;
     c.nblocks = g.nblocks;
@@ -216,22 +218,25 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
 struct StageLayout {
     uint32_t mask, rank, low, smhi, sm, raw, expanded, cap, bytes;
 };
-__host__ __device__ inline StageLayout make_stage_layout(int dt, int m, int hbits) {
+constexpr uint32_t kStageRankTable = kStageBytes - kRankTableBytes;  // where a stage keeps a stream's rank table
+// mapped: the stage also holds the stream's rank -> exponent table (its last 256 bytes).
+__host__ __device__ inline StageLayout make_stage_layout(int dt, int m, int hbits, bool mapped = false) {
     StageLayout L;
+    const uint32_t usable = mapped ? kStageRankTable : kStageBytes;
     L.mask = kStageMetaBytes;
     L.rank = L.mask + kGroupsPerBlock / 8;
     L.low = L.rank + kGroupsPerBlock * 2;
     L.smhi = L.low + kBlockElems * uint32_t(m) / 8;
     L.sm = L.smhi + (dt == ENEC_FP16 ? kBlockElems * 3 / 8 : 0);
     L.raw = L.sm + kBlockElems;  // at most 35072 (m = 8, or fp16 with m = 5), so a stage always has room
-    uint32_t cap = hbits > 0 ? (kStageBytes - L.raw - 64) / uint32_t(2 * hbits + 16) : 0;
+    uint32_t cap = hbits > 0 ? (usable - L.raw - 64) / uint32_t(2 * hbits + 16) : 0;
     if (cap > kGroupsPerBlock) cap = kGroupsPerBlock;
     L.cap = cap;
     L.expanded = L.raw + uint32_t(align16(uint64_t(cap) * 2 * hbits + 32));
     L.bytes = L.expanded + (cap + 1) * 16;
     return L;
 }
-static_assert(kStageMetaBytes + kGroupsPerBlock / 8 + kGroupsPerBlock * 2 + 2 * kBlockElems + 64 <= kStageBytes,
+static_assert(kStageMetaBytes + kGroupsPerBlock / 8 + kGroupsPerBlock * 2 + 2 * kBlockElems + 64 + kRankTableBytes <= kStageBytes,
               "the fixed part of the widest block fits a stage");
 
 struct RunCtx {
@@ -245,7 +250,8 @@ struct RunCtx {
     uint32_t real;        // real elements in the block
     uint32_t c4_or_h, fix, s4, b4;  // packed transform constants
     uint32_t c4;                    // rep4(b + 2^(n-1)) when that sum fits a byte
-    int n;
+    int n;                          // 0 marks the frequency-rank variant: c4 is then the shared address of the
+                                    // stage's rank -> exponent table, and the general body looks values up in it
 };
 
 // Inverse transform on four packed bytes: x = (b - sext_n(y)) mod 2^E  (Sec. 5.3).
@@ -264,6 +270,13 @@ __device__ __forceinline__ uint32_t inverse_transform4(const RunCtx& r, uint32_t
     }
     if (DT == ENEC_FP16) x &= 0x1F1F1F1Fu;
     return x;
+}
+
+// Four table look-ups (frequency-rank variant): byte i of the result is the exponent of the rank in byte i of y.
+__device__ __forceinline__ uint32_t table4(uint32_t table, uint32_t y) {
+    const uint32_t r0 = lds8(table + (y & 0xFFu)), r1 = lds8(table + ((y >> 8) & 0xFFu));
+    const uint32_t r2 = lds8(table + ((y >> 16) & 0xFFu)), r3 = lds8(table + (y >> 24));
+    return r0 | (r1 << 8) | (r2 << 16) | (r3 << 24);
 }
 
 // High bits of eight elements of a wide group whose record was not expanded in shared memory.
@@ -305,8 +318,8 @@ __device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, u
             y.y |= hi.y << M;
         }
     }
-    const uint32_t x0 = inverse_transform4<DT>(r, y.x);
-    const uint32_t x1 = inverse_transform4<DT>(r, y.y);
+    const uint32_t x0 = r.n == 0 ? table4(r.c4, y.x) : inverse_transform4<DT>(r, y.x);
+    const uint32_t x1 = r.n == 0 ? table4(r.c4, y.y) : inverse_transform4<DT>(r, y.y);
     const uint2 smv = lds64(r.sm + e0);
     uint32_t lo0, lo1, hi0, hi1;
     if (DT != ENEC_FP16) {
@@ -599,7 +612,7 @@ struct BlockDesc {
     uint32_t expect;    // wide groups of the block according to the prefix table
     uint32_t N;         // padded block length
     uint32_t real;      // real elements
-    uint32_t code;      // m * 8 + (n - m)
+    uint32_t code;      // m * 8 + (n - m); bit 8: frequency-rank variant (the stage then holds the rank table)
     uint32_t b, n;
     StageLayout L;
     uint16_t* out;        // global: first element of the block
@@ -649,7 +662,7 @@ __device__ __forceinline__ void prefetch_before_wait(const DecodeBatch& batch, u
     if (h0.x != kMagic || n < 1 || n > exp_bits(DT) || m < 1 || m > n) return;
     const Geometry g = make_geometry(job.count);
     if (k >= g.nblocks) return;
-    const Sections sec = make_sections(DT, job.count, g, n, m, h2.x);
+    const Sections sec = make_sections(DT, job.count, g, n, m, h2.x, (h0.y >> 24) == 1);
     if (sec.total > job.in_size) return;
     const uint32_t* table = reinterpret_cast<const uint32_t*>(job.in + sec.table);
     const uint32_t ahead = n_mine < kStages ? n_mine : kStages;
@@ -768,10 +781,14 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                     break;
                 }
                 hbits = jc.n - jc.m;
-                L = make_stage_layout(DT, jc.m, hbits);
+                L = make_stage_layout(DT, jc.m, hbits, jc.mapped);
                 table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
                 t0 = e0;
                 t1 = e1;
+                if (jc.mapped) {  // the table of a frequency-rank stream sits behind its rank table
+                    t0 = table[k];
+                    t1 = table[k + 1];
+                }
                 parsed = true;
             } else {
                 t0 = t1;
@@ -805,7 +822,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             d->expect = t1 - t0;
             d->N = N;
             d->real = real;
-            d->code = uint32_t(jc.m * 8 + hbits);
+            d->code = uint32_t(jc.m * 8 + hbits) | (jc.mapped ? 256u : 0u);
             d->b = uint32_t(jc.b);
             d->n = uint32_t(jc.n);
             d->L = L;
@@ -820,7 +837,9 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                 d->lo = nullptr;
             }
             d->high = jc.in + h0;
-            mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes);
+            mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes +
+                                              (jc.mapped ? kRankTableBytes : 0u));
+            if (jc.mapped) bulk_g2s(st + kStageRankTable, jc.in + kHeaderBytes, kRankTableBytes, &ctl->full[s]);
             bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
             bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
             if (DT == ENEC_FP16)
@@ -860,7 +879,8 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                        o_exp = d->L.expanded;
         const uint32_t sbit = 1u << (n - 1);
         const bool simple_sub = DT == ENEC_FP16 || n == 8 || b + sbit <= 255;
-        const bool full_block = N == kBlockElems && d->real == kBlockElems && expect <= cap && simple_sub;
+        const bool mapped = (code & 256u) != 0;   // ranks go through the general body: the branch-free one is built on the subtraction
+        const bool full_block = N == kBlockElems && d->real == kBlockElems && expect <= cap && simple_sub && !mapped;
         // preparation: ranks of the wide groups and expanded records
         if (hbits > 0) {
             // the branch-free body wants narrow groups to point at the flip slot and flipped records
@@ -889,10 +909,14 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             r.out = d->out;
             r.high = d->high;
             r.lo = d->lo;
+            if (mapped) {
+                r.n = 0;
+                r.c4 = st + kStageRankTable;
+            }
             r.real = d->real;
         }
         if (consumer_barrier_or(*abort_flag != 0)) break;
-        switch (code) {
+        switch (code & 255u) {
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
         if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid);     \

@@ -32,6 +32,8 @@ struct alignas(16) EncodeControl {
     uint32_t hist_done;            // CTAs of the histogram kernel that have finished
     uint32_t reserved;
     int b, n, m;                   // result of the parameter search
+    uint8_t lut[256];              // frequency-rank variant: exponent -> rank
+    uint8_t unmap[256];            // frequency-rank variant: rank -> exponent (goes into the stream)
 };
 static_assert(sizeof(EncodeControl) <= kControlSlotBytes, "a control set fits its slot");
 
@@ -61,6 +63,7 @@ struct EncodeJob {
     int b, n, m;                   // used when from_search == 0
     int from_search;               // take (b, n, m) from ctl
     int check;                     // verify that (b, n) keeps every exponent
+    int ranked;                    // frequency-rank variant: stored value = ctl->lut[exponent]
 };
 
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
@@ -130,6 +133,28 @@ __host__ __device__ inline int width_eq1(int b, int l, int h, int E) {
     return n;
 }
 
+// Eq. 4 at L = 16 for every m in 1..n, given the number of elements per bit width of the stored value; one
+// thread. Plain IEEE double, one rounding per operation, no fused multiply-add; ties go to the smaller m.
+__device__ inline int choose_m(const unsigned long long* width_count, int n) {
+    unsigned long long total = 0;
+    for (int w = 0; w <= 8; ++w) total += width_count[w];
+    unsigned long long cnt = width_count[0];
+    int best_m = 1;
+    double best_bits = 0.0;
+    for (int m = 1; m <= n; ++m) {
+        cnt += width_count[m];
+        const double p = __ddiv_rn(__ull2double_rn(cnt), __ull2double_rn(total));
+        const double p2 = __dmul_rn(p, p);
+        const double p4 = __dmul_rn(p2, p2);
+        const double p8 = __dmul_rn(p4, p4);
+        const double p16 = __dmul_rn(p8, p8);
+        const double saving = __dmul_rn(double(m - n), p16);
+        const double bits = __dadd_rn(__dadd_rn(double(n), 0.0625), saving);  // 1/L + n + (m - n) p^L
+        if (m == 1 || bits < best_bits) { best_m = m; best_bits = bits; }
+    }
+    return best_m;
+}
+
 // Sec. 5.5 phases 2 and 3 on the finished histogram; all kHistThreads threads of one CTA.
 template <int DT>
 __device__ void parameter_search(EncodeControl* ctl) {
@@ -179,30 +204,48 @@ __device__ void parameter_search(EncodeControl* ctl) {
     }
     __syncthreads();
     if (tid == 0) {
-        unsigned long long total = 0;
-        for (int w = 0; w <= 8; ++w) total += s_width_count[w];
-        unsigned long long cnt = s_width_count[0];
-        int best_m = 1;
-        double best_bits = 0.0;
-        for (int m = 1; m <= n; ++m) {
-            cnt += s_width_count[m];
-            // plain IEEE double, one rounding per operation, no fused multiply-add
-            const double p = __ddiv_rn(__ull2double_rn(cnt), __ull2double_rn(total));
-            const double p2 = __dmul_rn(p, p);
-            const double p4 = __dmul_rn(p2, p2);
-            const double p8 = __dmul_rn(p4, p4);
-            const double p16 = __dmul_rn(p8, p8);
-            const double saving = __dmul_rn(double(m - n), p16);
-            const double bits = __dadd_rn(__dadd_rn(double(n), 0.0625), saving);  // 1/L + n + (m - n) p^L
-            if (m == 1 || bits < best_bits) { best_m = m; best_bits = bits; }
-        }
         ctl->b = b;
         ctl->n = n;
-        ctl->m = best_m;
+        ctl->m = choose_m(s_width_count, n);
     }
 }
 
+// The frequency-rank variant (Sec. 4.2, Algorithm 1): exponents sorted by falling count (ties: smaller exponent
+// first) give the codes 0, 1, 2, ...; n = bits of the largest code, m by Eq. 4 over the codes' bit widths.
 template <int DT>
+__device__ void parameter_search_ranked(EncodeControl* ctl) {
+    constexpr int kBins = 1 << HistShape<DT>::E;
+    __shared__ unsigned long long s_hist[256];
+    __shared__ unsigned long long s_width_count[9];
+    __shared__ uint32_t s_occupied;
+    const uint32_t tid = threadIdx.x;
+    s_hist[tid] = tid < uint32_t(kBins) ? ld_relaxed_u64(&ctl->hist[tid]) : 0ull;
+    if (tid < 9) s_width_count[tid] = 0;
+    if (tid == 0) s_occupied = 0;
+    ctl->unmap[tid] = 0;
+    __syncthreads();
+    const unsigned long long mine = s_hist[tid];
+    uint32_t rank = 0;
+    if (mine) {
+        for (uint32_t u = 0; u < uint32_t(kBins); ++u) {
+            const unsigned long long other = s_hist[u];
+            rank += (other > mine || (other == mine && u < tid)) ? 1u : 0u;
+        }
+        atomicAdd(&s_occupied, 1u);
+        atomicAdd(&s_width_count[bit_width_u32(rank)], mine);
+    }
+    ctl->lut[tid] = uint8_t(rank);
+    __syncthreads();
+    if (mine) ctl->unmap[rank] = uint8_t(tid);
+    if (tid == 0) {
+        const int n = s_occupied <= 1 ? 1 : bit_width_u32(s_occupied - 1);
+        ctl->b = 0;
+        ctl->n = n;
+        ctl->m = choose_m(s_width_count, n);
+    }
+}
+
+template <int DT, bool RANKED = false>
 __global__ void __launch_bounds__(kHistThreads, 3)
 enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeControl* ctl) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -286,7 +329,8 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    parameter_search<DT>(ctl);
+    if constexpr (RANKED) parameter_search_ranked<DT>(ctl);
+    else parameter_search<DT>(ctl);
 }
 
 // Histograms of a list of tensors in one launch. The tensors are cut into units of at most kHistUnitChunks
@@ -570,7 +614,15 @@ struct TransformCtx {
     uint32_t s4;        // rep4(2^(n-1))
     uint32_t emask4;    // rep4(2^E - 1)
     int n, E;
+    uint32_t lut;       // frequency-rank variant: shared address of the exponent -> rank table, else 0
 };
+
+// Four table look-ups: byte i of the result is the table entry of byte i of v.
+__device__ __forceinline__ uint32_t lut4(uint32_t table, uint32_t v) {
+    const uint32_t r0 = lds8(table + (v & 0xFFu)), r1 = lds8(table + ((v >> 8) & 0xFFu));
+    const uint32_t r2 = lds8(table + ((v >> 16) & 0xFFu)), r3 = lds8(table + (v >> 24));
+    return r0 | (r1 << 8) | (r2 << 16) | (r3 << 24);
+}
 
 // b - x modulo 256 in every byte
 __device__ __forceinline__ uint32_t bytewise_b_minus(const TransformCtx& t, uint32_t x) {
@@ -622,7 +674,7 @@ __device__ __forceinline__ uint4 load_fp32_run(const uint8_t* __restrict__ p, ui
 // Returns the wide flags of the thread's eight runs (bit c).
 // With DT = ENEC_FP32 the values are 32-bit words: their high halves take bf16's path, their low halves are
 // stored as they are to `lo_thread` (two bytes per value).
-template <int DT, bool SIMPLE>
+template <int DT, bool SIMPLE, bool RANKED = false>
 __device__ __forceinline__ uint32_t encode_full_runs(const uint8_t* in_thread, uint8_t* sm_thread, uint8_t* lo_thread,
                                                      const TransformCtx& tc, int m, uint32_t warp, uint32_t lane,
                                                      uint32_t* mask_words, uint2 (&y)[8], uint2 (&hs)[8], int& bad) {
@@ -661,10 +713,14 @@ __device__ __forceinline__ uint32_t encode_full_runs(const uint8_t* in_thread, u
         } else {
             const Split4 s0 = split4<DT>(raw[c].x, raw[c].y);
             const Split4 s1 = split4<DT>(raw[c].z, raw[c].w);
-            const uint32_t d0 = bytewise_b_minus(tc, s0.x), d1 = bytewise_b_minus(tc, s1.x);
-            y[c] = make_uint2(d0 & tc.nmask4, d1 & tc.nmask4);
+            if constexpr (RANKED) {  // frequency-rank variant: the stored value is the exponent's rank
+                y[c] = make_uint2(lut4(tc.lut, s0.x), lut4(tc.lut, s1.x));
+            } else {
+                const uint32_t d0 = bytewise_b_minus(tc, s0.x), d1 = bytewise_b_minus(tc, s1.x);
+                y[c] = make_uint2(d0 & tc.nmask4, d1 & tc.nmask4);
+                bad |= (lossy_bytes(tc, d0, y[c].x) | lossy_bytes(tc, d1, y[c].y)) != 0;
+            }
             hs[c] = make_uint2(s0.hs, s1.hs);
-            bad |= (lossy_bytes(tc, d0, y[c].x) | lossy_bytes(tc, d1, y[c].y)) != 0;
             sm0 = s0.sm;
             sm1 = s1.sm;
         }
@@ -707,8 +763,8 @@ __device__ __noinline__ int encode_short_block(const uint16_t* in, uint32_t N, u
         if (DT != ENEC_FP16) { x = (w >> 7) & 0xFF; sm = ((w >> 8) & 0x80) | (w & 0x7F); }
         else { x = (w >> 10) & 0x1F; sm = w & 0xFF; hs = ((w >> 13) & 4) | ((w >> 8) & 3); }
         if (tid < real) {
-            y = uint32_t(b - int(x)) & ((1u << n) - 1);
-            if (check && n < tc.E) {
+            y = tc.lut ? lds8(tc.lut + x) : uint32_t(b - int(x)) & ((1u << n) - 1);
+            if (check && n < tc.E && !tc.lut) {
                 const int v = (y >> (n - 1)) ? int(y) - (1 << n) : int(y);
                 bad = (uint32_t(b - v) & ((1u << tc.E) - 1)) != x;
             }
@@ -777,7 +833,7 @@ struct EncodeTensor {
 // address `rec`, `wide_count` of them) to their place in the stream and write its table entry; the last
 // block also writes the header, the end of the table and the stream length. The look-back is done by
 // warp 0, up to 256 words per round trip, down to the nearest block that already knows its prefix.
-template <int DT>
+template <int DT, bool RANKED = false>
 __device__ __forceinline__ void resolve_block(const EncodeJob& job, const EncodeTensor& t, uint32_t k, uint32_t wide_count,
                                               bool own_taint, const uint8_t* rec, EncodeShared& sh, int* status) {
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -864,6 +920,9 @@ __device__ __forceinline__ void resolve_block(const EncodeJob& job, const Encode
         for (uint32_t i = tid; i < wide_count * hbits; i += kEncodeThreads) dst[i] = src[i];
         if (tid == 0) table[k] = before;
     }
+    if constexpr (RANKED) {
+        if (k + 1 == t.g.nblocks) job.out[t.sec.unmap + tid] = job.ctl->unmap[tid];  // 256 threads, 256 bytes
+    }
     if (k + 1 == t.g.nblocks && tid == 0) {
         const uint32_t a_total = before + wide_count;
         const uint64_t high_bytes = uint64_t(a_total) * 2 * hbits;
@@ -873,7 +932,7 @@ __device__ __forceinline__ void resolve_block(const EncodeJob& job, const Encode
         hd.magic = failed ? 0 : kMagic;
         hd.version = kVersion;
         hd.dtype = DT;
-        hd.pad0 = 0;
+        hd.variant = RANKED ? 1 : 0;
         hd.count = job.count;
         hd.block = kBlockElems;
         hd.b = uint8_t(t.b); hd.n = uint8_t(t.n); hd.m = uint8_t(t.m); hd.L = kGroupElems;
@@ -912,13 +971,13 @@ struct BlockCtx {
     uint32_t k;  // block index inside the tensor
 };
 
-template <int DT>
+template <int DT, bool RANKED = false>
 __device__ __forceinline__ void fill_tensor_ctx(const EncodeJob& job, EncodeTensor& tensor, TransformCtx& tc) {
     constexpr int E = DT == ENEC_FP16 ? 5 : 8;
     int b = job.b, n = job.n, m = job.m;
     if (job.from_search) { b = job.ctl->b; n = job.ctl->n; m = job.ctl->m; }
     tensor.g = make_geometry(job.count);
-    tensor.sec = make_sections(DT, job.count, tensor.g, n, m, 0);
+    tensor.sec = make_sections(DT, job.count, tensor.g, n, m, 0, RANKED);
     tensor.b = b; tensor.n = n; tensor.m = m; tensor.hbits = n - m;
     tc.b4 = rep4(uint32_t(b));
     tc.b4_or_h = tc.b4 | 0x80808080u;
@@ -927,10 +986,13 @@ __device__ __forceinline__ void fill_tensor_ctx(const EncodeJob& job, EncodeTens
     tc.emask4 = rep4((1u << E) - 1);
     tc.n = n;
     tc.E = E;
+    tc.lut = 0;
 }
 
 // BATCH = false: one tensor, described by `single`. BATCH = true: the tensors of `batch`; `single` is unused.
-template <int DT, bool BATCH>
+// RANKED (one tensor only): the frequency-rank variant; a separate instance, so that the usual one carries
+// nothing of the table look-ups.
+template <int DT, bool BATCH, bool RANKED = false>
 __global__ void __launch_bounds__(kEncodeThreads, 4)
 enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status) {
     // dynamic shared memory: low plane | fp16 sign/mantissa-high plane | two record buffers
@@ -943,6 +1005,7 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
     pdl_launch_dependents();
     pdl_wait();  // nothing above touches global memory
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ uint8_t s_lut[RANKED ? 256 : 1];
     __shared__ BlockCtx s_ctx[BATCH ? 3 : 1];  // batched: this block's, the previous block's and the next block's tensor
     EncodeTensor single_tensor{};
     TransformCtx single_tc{};
@@ -951,7 +1014,11 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
             single.ctl_next->hist[tid] = 0;
             if (tid == 0) { single.ctl_next->ticket = 0; single.ctl_next->hist_done = 0; }
         }
-        fill_tensor_ctx<DT>(single, single_tensor, single_tc);
+        fill_tensor_ctx<DT, RANKED>(single, single_tensor, single_tc);
+        if constexpr (RANKED) {  // the exponent -> rank table of the tensor, for every block of this CTA
+            s_lut[tid] = single.ctl->lut[tid];
+            single_tc.lut = smem_u32(s_lut);
+        }
     }
     uint32_t* const ticket = BATCH ? batch.ticket : &single.ctl->ticket;
     const uint32_t total_blocks = BATCH ? batch.total_blocks : single_tensor.g.nblocks;
@@ -1021,10 +1088,10 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
 
     uint2 hs[8];
     if (fast) {
-        if (!job.check && n < 8)
+        if (!RANKED && !job.check && n < 8)
             wide_bits = encode_full_runs<DT, true>(in_bytes + j * kElemBytes, out_sm + j, out_smlo + j * 2, tc, m, warp, lane, sh.mask, y, hs, bad);
         else
-            wide_bits = encode_full_runs<DT, false>(in_bytes + j * kElemBytes, out_sm + j, out_smlo + j * 2, tc, m, warp, lane, sh.mask, y, hs, bad);
+            wide_bits = encode_full_runs<DT, false, RANKED>(in_bytes + j * kElemBytes, out_sm + j, out_smlo + j * 2, tc, m, warp, lane, sh.mask, y, hs, bad);
         uint2 ylow[8];
         const uint32_t lowmask4 = rep4((1u << m) - 1);
 #pragma unroll
@@ -1070,8 +1137,14 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
             const uint32_t e0 = c * n8 + j;
             const Split4 s0 = split4<DT>(raw[c].x, raw[c].y);
             const Split4 s1 = split4<DT>(raw[c].z, raw[c].w);
-            const uint32_t d0 = bytewise_b_minus(tc, s0.x), d1 = bytewise_b_minus(tc, s1.x);
-            y[c] = make_uint2(d0 & tc.nmask4, d1 & tc.nmask4);
+            uint32_t d0 = 0, d1 = 0;
+            if constexpr (RANKED) {  // frequency-rank variant (never with job.check)
+                y[c] = make_uint2(lut4(tc.lut, s0.x), lut4(tc.lut, s1.x));
+            } else {
+                d0 = bytewise_b_minus(tc, s0.x);
+                d1 = bytewise_b_minus(tc, s1.x);
+                y[c] = make_uint2(d0 & tc.nmask4, d1 & tc.nmask4);
+            }
             hs[c] = make_uint2(s0.hs, s1.hs);
             if (active && e0 + 8 > real) {  // padding elements carry y = 0
                 const uint32_t valid = e0 < real ? real - e0 : 0;
@@ -1192,7 +1265,7 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
     // the previous block of this CTA, whose records wait in the other buffer
     if (pending_block != 0xFFFFFFFFu) {
         const BlockCtx& px = s_ctx[BATCH ? (iter + 2) % 3 : 0];
-        resolve_block<DT>(BATCH ? px.job : single, BATCH ? px.tensor : single_tensor, pending_block, pending_wide, pending_bad,
+        resolve_block<DT, RANKED>(BATCH ? px.job : single, BATCH ? px.tensor : single_tensor, pending_block, pending_wide, pending_bad,
                           s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
     }
     pending_block = k;
@@ -1202,19 +1275,21 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
     }
     if (pending_block != 0xFFFFFFFFu) {
         const BlockCtx& px = s_ctx[BATCH ? (iter + 2) % 3 : 0];
-        resolve_block<DT>(BATCH ? px.job : single, BATCH ? px.tensor : single_tensor, pending_block, pending_wide, pending_bad,
+        resolve_block<DT, RANKED>(BATCH ? px.job : single, BATCH ? px.tensor : single_tensor, pending_block, pending_wide, pending_bad,
                           s_rec_base + (cur ^ 1) * EncodeSmem<DT>::kRecBytes, sh, status);
     }
 }
 
-// Stream of an empty tensor: header and a one-entry table.
-__global__ void enec_encode_empty_kernel(uint8_t* out, int dt, int b, int n, int m, unsigned long long* out_size) {
+// Stream of an empty tensor: header, (frequency-rank variant: an all-zero rank table) and a one-entry table.
+__global__ void enec_encode_empty_kernel(uint8_t* out, int dt, int b, int n, int m, unsigned long long* out_size,
+                                         int ranked = 0) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const uint32_t table_at = kHeaderBytes + (ranked ? kRankTableBytes : 0);
     Header hd;
     hd.magic = kMagic;
     hd.version = kVersion;
     hd.dtype = uint8_t(dt);
-    hd.pad0 = 0;
+    hd.variant = ranked ? 1 : 0;
     hd.count = 0;
     hd.block = kBlockElems;
     hd.b = uint8_t(b); hd.n = uint8_t(n); hd.m = uint8_t(m); hd.L = kGroupElems;
@@ -1222,11 +1297,11 @@ __global__ void enec_encode_empty_kernel(uint8_t* out, int dt, int b, int n, int
     hd.total_groups = 0;
     hd.a_total = 0;
     hd.pad1 = 0;
-    hd.total_bytes = kHeaderBytes + 16;
+    hd.total_bytes = table_at + 16;
     hd.pad2[0] = hd.pad2[1] = 0;
     *reinterpret_cast<Header*>(out) = hd;
-    *reinterpret_cast<uint4*>(out + kHeaderBytes) = make_uint4(0, 0, 0, 0);
-    if (out_size) *out_size = kHeaderBytes + 16;
+    for (uint32_t at = kHeaderBytes; at <= table_at; at += 16) *reinterpret_cast<uint4*>(out + at) = make_uint4(0, 0, 0, 0);
+    if (out_size) *out_size = table_at + 16;
 }
 
 }  // namespace enec

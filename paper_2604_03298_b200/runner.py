@@ -59,7 +59,8 @@ class CodecSet:
     def allocate(cls, raw: List[torch.Tensor], share_output: bool = False) -> "CodecSet":
         dev = raw[0].device
         cs = cls(raw=[t.contiguous() for t in raw])
-        cs.streams = [torch.empty(enec.enec_max_compressed_size(_DT[t.dtype], t.numel()), dtype=torch.uint8, device=dev)
+        # room for either variant of the stream (the frequency-rank variant is 256 bytes longer)
+        cs.streams = [torch.empty(enec.enec_max_compressed_size_ranked(_DT[t.dtype], t.numel()), dtype=torch.uint8, device=dev)
                       for t in cs.raw]
         cs.shared_outs = share_output
         if share_output:
@@ -104,15 +105,18 @@ class CodecSet:
             done.record(s)
             main.wait_event(done)
 
-    def compress_all(self, params=None, n_streams: int = 1) -> None:
+    def compress_all(self, params=None, n_streams: int = 1, ranked: bool = False) -> None:
         """One enec_compress per tensor (no host synchronisation), on the current stream or spread over
-        n_streams side streams."""
-        self.spread(n_streams, lambda i: self._compress_one(i, params))
+        n_streams side streams. ranked: the frequency-rank variant (enec_compress_ranked) instead."""
+        self.spread(n_streams, lambda i: self._compress_one(i, params, ranked))
 
-    def _compress_one(self, i: int, params) -> None:
+    def _compress_one(self, i: int, params, ranked: bool = False) -> None:
         t = self.raw[i]
         dt = _DT[t.dtype]
-        if params is None:
+        if ranked:
+            st = enec.enec_compress_ranked(t, dt, t.numel(), self.streams[i], self.streams[i].numel(),
+                                           self.sizes[i:i + 1], self.status)
+        elif params is None:
             st = enec.enec_compress(t, dt, t.numel(), self.streams[i], self.streams[i].numel(),
                                     self.sizes[i:i + 1], self.status)
         else:
