@@ -97,13 +97,17 @@ enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, siz
  * of an element is the rank of its exponent when the tensor's exponents are sorted by falling count (ties:
  * smaller exponent first), n is the bit width of the largest rank and m follows Eq. 4; there is no base b and
  * no sign bit. The stream has header byte 7 = 1 and a 256-byte table (rank -> exponent) between the header and
- * the prefix table; everything else is laid out as by enec_compress. enec_decompress and
- * enec_decompress_batched read both kinds of stream. out_capacity must be at least
+ * the prefix table; everything else is laid out as by enec_compress. out_capacity must be at least
  * enec_max_compressed_size_ranked(dt, count) (256 bytes more than enec_max_compressed_size).
+ * Such a stream is decoded by enec_decompress_ranked (same arguments as enec_decompress); each of the two
+ * decompress calls reports ENEC_ERR_BAD_STREAM in *d_status for the other kind of stream, and
+ * enec_decompress_batched takes streams of enec_compress only.
  */
 size_t enec_max_compressed_size_ranked(enec_dtype dt, size_t count);
 enec_status enec_compress_ranked(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
                                  size_t* d_out_size, int* d_status, enec_stream_t stream);
+enec_status enec_decompress_ranked(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
+                                   int* d_status, enec_stream_t stream);
 
 /* One tensor of a batch. All pointers are device pointers. */
 typedef struct {

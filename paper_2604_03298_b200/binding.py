@@ -52,6 +52,8 @@ def lib():
         L.enec_decompress.argtypes = [C.c_void_p, C.c_size_t, C.c_int, C.c_size_t, C.c_void_p, C.c_void_p,
                                       C.c_void_p]
         L.enec_decompress.restype = C.c_int
+        L.enec_decompress_ranked.argtypes = L.enec_decompress.argtypes
+        L.enec_decompress_ranked.restype = C.c_int
         L.enec_decompress_batched.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.enec_decompress_batched.restype = C.c_int
         L.enec_compress_batched.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -116,6 +118,11 @@ def make_batch(items):
     for i, (src, dst, count, size) in enumerate(items):
         arr[i].d_in, arr[i].d_out, arr[i].count, arr[i].size = src.data_ptr(), dst.data_ptr(), count, size
     return arr
+
+
+def enec_decompress_ranked(d_in, in_size, dt, count, d_out, d_status=None) -> int:
+    """Decompresses a stream written by enec_compress_ranked."""
+    return lib().enec_decompress_ranked(_ptr(d_in), in_size, dt, count, _ptr(d_out), _ptr(d_status), _stream())
 
 
 def enec_decompress_batched(items, dt, d_status=None) -> int:

@@ -51,12 +51,14 @@ static cudaError_t launch_pdl(void (*kernel)(KernelArgs...), uint32_t grid, uint
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 template <int DT>
-static enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream) {
+static enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked = false) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
     DeviceInfo& info = device_info(dev);
     if (!info.decode_attr_set[DT]) {
-        if (cudaFuncSetAttribute(enec_decode_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(enec_decode_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(kDecodeSmemBytes)) != cudaSuccess ||
+            cudaFuncSetAttribute(enec_decode_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(kDecodeSmemBytes)) != cudaSuccess)
             return ENEC_ERR_CUDA;
         info.decode_attr_set[DT] = true;
@@ -64,7 +66,9 @@ static enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaSt
     uint32_t grid = uint32_t(info.sms) * 3;  // three resident CTAs per SM
     if (grid > batch.total_blocks) grid = batch.total_blocks;
     if (grid == 0) grid = 1;
-    const cudaError_t err = launch_pdl(enec_decode_kernel<DT>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status);
+    const cudaError_t err =
+        ranked ? launch_pdl(enec_decode_kernel<DT, true>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status)
+               : launch_pdl(enec_decode_kernel<DT, false>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
@@ -302,8 +306,8 @@ size_t enec_max_compressed_size(enec_dtype dt, size_t count) {
     return size_t(worst);
 }
 
-enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
-                            int* d_status, enec_stream_t stream) {
+static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
+                                  int* d_status, cudaStream_t stream, bool ranked) {
     if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if (!d_in || (!d_out && count) || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out))
         return ENEC_ERR_INVALID_ARG;
@@ -317,9 +321,19 @@ enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, siz
                                      uint64_t(in_size)};
     batch.inline_prefix[0] = 0;
     batch.inline_prefix[1] = batch.total_blocks;
-    return dt == ENEC_BF16   ? launch_decode<ENEC_BF16>(batch, d_status, stream)
-           : dt == ENEC_FP16 ? launch_decode<ENEC_FP16>(batch, d_status, stream)
-                             : launch_decode<ENEC_FP32>(batch, d_status, stream);
+    return dt == ENEC_BF16   ? launch_decode<ENEC_BF16>(batch, d_status, stream, ranked)
+           : dt == ENEC_FP16 ? launch_decode<ENEC_FP16>(batch, d_status, stream, ranked)
+                             : launch_decode<ENEC_FP32>(batch, d_status, stream, ranked);
+}
+
+enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
+                            int* d_status, enec_stream_t stream) {
+    return decompress_one(d_in, in_size, dt, count, d_out, d_status, stream, false);
+}
+
+enec_status enec_decompress_ranked(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
+                                   int* d_status, enec_stream_t stream) {
+    return decompress_one(d_in, in_size, dt, count, d_out, d_status, stream, true);
 }
 
 enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, int* d_status,

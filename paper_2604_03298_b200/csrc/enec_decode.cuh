@@ -177,12 +177,11 @@ struct JobCtx {
     uint32_t nblocks, tail_real, tail_padded;
     uint32_t a_total;
     int b, n, m;
-    bool mapped;  // frequency-rank variant: the stored value is a rank, looked up in the stream's table (behind the header)
     uint64_t off_table, off_mask, off_low, off_smhi, off_sm, off_smlo, off_high, total;
 };
 
 // Reads and validates the header. Returns 0 or an enec_status.
-template <int DT>
+template <int DT, bool MAPPED = false>
 __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
     if (job.in_size < kHeaderBytes + 16) return ENEC_ERR_BAD_STREAM;
     const Header h = *reinterpret_cast<const Header*>(job.in);
@@ -190,13 +189,12 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
         h.block != kBlockElems || h.L != kGroupElems)
         return ENEC_ERR_BAD_STREAM;
     constexpr int E = exp_bits(DT);
-    if (h.n < 1 || h.n > E || h.m < 1 || h.m > h.n || h.b >= (1 << E) || h.variant > 1) return ENEC_ERR_BAD_STREAM;
+    if (h.n < 1 || h.n > E || h.m < 1 || h.m > h.n || h.b >= (1 << E) || h.variant != (MAPPED ? 1 : 0)) return ENEC_ERR_BAD_STREAM;
     const Geometry g = make_geometry(job.count);
     if (h.nblocks != g.nblocks || h.total_groups != g.total_groups || h.a_total > g.total_groups)
         return ENEC_ERR_BAD_STREAM;
-    const Sections s = make_sections(DT, job.count, g, h.n, h.m, h.a_total, h.variant == 1);
+    const Sections s = make_sections(DT, job.count, g, h.n, h.m, h.a_total, MAPPED);
     if (h.total_bytes != s.total || job.in_size < s.total) return ENEC_ERR_BAD_STREAM;
-    c.mapped = h.variant == 1;
     c.in = job.in;
     c.out = job.out;
     c.nblocks = g.nblocks;
@@ -250,8 +248,7 @@ struct RunCtx {
     uint32_t real;        // real elements in the block
     uint32_t c4_or_h, fix, s4, b4;  // packed transform constants
     uint32_t c4;                    // rep4(b + 2^(n-1)) when that sum fits a byte
-    int n;                          // 0 marks the frequency-rank variant: c4 is then the shared address of the
-                                    // stage's rank -> exponent table, and the general body looks values up in it
+    int n;
 };
 
 // Inverse transform on four packed bytes: x = (b - sext_n(y)) mod 2^E  (Sec. 5.3).
@@ -306,7 +303,7 @@ __device__ __forceinline__ void store_fp32_run(uint32_t* out, uint4 w, uint4 lo)
 
 // Finishes eight consecutive elements e0 .. e0+7 of a block: high bits of wide groups, inverse transform,
 // rejoin with sign/mantissa, store.
-template <int DT, int M, int HB>
+template <int DT, int M, int HB, bool MAPPED = false>
 __device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, uint32_t e0, bool active) {
     if constexpr (HB > 0) {
         const uint32_t rk = lds16(r.rank + ((e0 >> 4) << 1));
@@ -318,8 +315,9 @@ __device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, u
             y.y |= hi.y << M;
         }
     }
-    const uint32_t x0 = r.n == 0 ? table4(r.c4, y.x) : inverse_transform4<DT>(r, y.x);
-    const uint32_t x1 = r.n == 0 ? table4(r.c4, y.y) : inverse_transform4<DT>(r, y.y);
+    // frequency-rank variant: r.c4 is the shared address of the stage's rank -> exponent table
+    const uint32_t x0 = MAPPED ? table4(r.c4, y.x) : inverse_transform4<DT>(r, y.x);
+    const uint32_t x1 = MAPPED ? table4(r.c4, y.y) : inverse_transform4<DT>(r, y.y);
     const uint2 smv = lds64(r.sm + e0);
     uint32_t lo0, lo1, hi0, hi1;
     if (DT != ENEC_FP16) {
@@ -364,7 +362,7 @@ __device__ __forceinline__ void finish_run(const RunCtx& r, uint2 y, uint2 hs, u
 }
 
 // One block, all consumer threads. tid = 0..255. N = padded block length.
-template <int DT, int M, int HB>
+template <int DT, int M, int HB, bool MAPPED = false>
 __device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, uint32_t s_smhi, uint32_t N,
                                              uint32_t tid) {
     if (N >= 128) {
@@ -380,7 +378,7 @@ __device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, ui
             if (DT == ENEC_FP16) unpack_plane<3>(s_smhi, j, N, hs);
 #pragma unroll
             for (int c = 0; c < 8; ++c)
-                finish_run<DT, M, HB>(r, y[c], DT == ENEC_FP16 ? hs[c] : make_uint2(0, 0), c * n8 + j, active);
+                finish_run<DT, M, HB, MAPPED>(r, y[c], DT == ENEC_FP16 ? hs[c] : make_uint2(0, 0), c * n8 + j, active);
         }
     } else {
         // short tail block (16, 32 or 64 elements): one run of eight per thread, values rebuilt bit by bit
@@ -392,7 +390,7 @@ __device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, ui
             if (DT == ENEC_FP16)
                 hb[i >> 2] |= unpack_scalar([&](uint32_t p) { return lds8(s_smhi + p); }, N, 3, e0 + i) << (8 * (i & 3));
         }
-        finish_run<DT, M, HB>(r, make_uint2(yb[0], yb[1]), make_uint2(hb[0], hb[1]), e0, true);
+        finish_run<DT, M, HB, MAPPED>(r, make_uint2(yb[0], yb[1]), make_uint2(hb[0], hb[1]), e0, true);
     }
 }
 
@@ -647,7 +645,7 @@ __device__ __forceinline__ uint4 ldg_l2_only(const void* p) {
 // used for anything but prefetch addresses, every address stays inside the caller's buffer
 // [in, in + in_size), and the loads bypass L1; L2 is coherent, so a line prefetched too early is simply
 // updated by the writer. Only for tensor lists that travel in the kernel parameters.
-template <int DT>
+template <int DT, bool MAPPED = false>
 __device__ __forceinline__ void prefetch_before_wait(const DecodeBatch& batch, uint32_t first_block, uint32_t n_mine) {
     if (batch.jobs != nullptr || n_mine == 0) return;
     uint32_t j = 0;
@@ -662,7 +660,7 @@ __device__ __forceinline__ void prefetch_before_wait(const DecodeBatch& batch, u
     if (h0.x != kMagic || n < 1 || n > exp_bits(DT) || m < 1 || m > n) return;
     const Geometry g = make_geometry(job.count);
     if (k >= g.nblocks) return;
-    const Sections sec = make_sections(DT, job.count, g, n, m, h2.x, (h0.y >> 24) == 1);
+    const Sections sec = make_sections(DT, job.count, g, n, m, h2.x, MAPPED);
     if (sec.total > job.in_size) return;
     const uint32_t* table = reinterpret_cast<const uint32_t*>(job.in + sec.table);
     const uint32_t ahead = n_mine < kStages ? n_mine : kStages;
@@ -690,7 +688,9 @@ __device__ __forceinline__ void prefetch_before_wait(const DecodeBatch& batch, u
     }
 }
 
-template <int DT>
+// MAPPED: the instance for streams of the frequency-rank variant (general block body with table look-ups only);
+// each instance refuses the other kind of stream.
+template <int DT, bool MAPPED = false>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
 enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -703,7 +703,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     const uint32_t first_block = uint32_t(uint64_t(blockIdx.x) * batch.total_blocks / gridDim.x);
     const uint32_t end_block = uint32_t(uint64_t(blockIdx.x + 1) * batch.total_blocks / gridDim.x);
     const uint32_t n_mine = end_block - first_block;
-    if (threadIdx.x == kConsumerWarps * 32) prefetch_before_wait<DT>(batch, first_block, n_mine);
+    if (threadIdx.x == kConsumerWarps * 32) prefetch_before_wait<DT, MAPPED>(batch, first_block, n_mine);
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(&ctl->full[s], 1);
@@ -717,7 +717,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     if (batch.total_blocks == 0) {  // nothing to decode: only check the header of a single empty tensor
         if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr && batch.n_jobs == 1) {
             JobCtx jc;
-            const int err = load_job<DT>(batch.inline_jobs[0], jc);
+            const int err = load_job<DT, MAPPED>(batch.inline_jobs[0], jc);
             if (err) report(status, err);
         }
         return;
@@ -773,7 +773,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                     e0 = tb[k];
                     e1 = tb[k + 1];
                 }
-                const int err = early ? load_job<DT>(job, jc) : ENEC_ERR_BAD_STREAM;
+                const int err = early ? load_job<DT, MAPPED>(job, jc) : ENEC_ERR_BAD_STREAM;
                 if (err) {
                     *abort_flag = 1;
                     report(status, err);
@@ -781,11 +781,11 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                     break;
                 }
                 hbits = jc.n - jc.m;
-                L = make_stage_layout(DT, jc.m, hbits, jc.mapped);
+                L = make_stage_layout(DT, jc.m, hbits, MAPPED);
                 table = reinterpret_cast<const uint32_t*>(jc.in + jc.off_table);
                 t0 = e0;
                 t1 = e1;
-                if (jc.mapped) {  // the table of a frequency-rank stream sits behind its rank table
+                if constexpr (MAPPED) {  // the table of a frequency-rank stream sits behind its rank table
                     t0 = table[k];
                     t1 = table[k + 1];
                 }
@@ -822,7 +822,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             d->expect = t1 - t0;
             d->N = N;
             d->real = real;
-            d->code = uint32_t(jc.m * 8 + hbits) | (jc.mapped ? 256u : 0u);
+            d->code = uint32_t(jc.m * 8 + hbits);
             d->b = uint32_t(jc.b);
             d->n = uint32_t(jc.n);
             d->L = L;
@@ -838,8 +838,8 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             }
             d->high = jc.in + h0;
             mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes +
-                                              (jc.mapped ? kRankTableBytes : 0u));
-            if (jc.mapped) bulk_g2s(st + kStageRankTable, jc.in + kHeaderBytes, kRankTableBytes, &ctl->full[s]);
+                                              (MAPPED ? kRankTableBytes : 0u));
+            if constexpr (MAPPED) bulk_g2s(st + kStageRankTable, jc.in + kHeaderBytes, kRankTableBytes, &ctl->full[s]);
             bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
             bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
             if (DT == ENEC_FP16)
@@ -879,8 +879,8 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                        o_exp = d->L.expanded;
         const uint32_t sbit = 1u << (n - 1);
         const bool simple_sub = DT == ENEC_FP16 || n == 8 || b + sbit <= 255;
-        const bool mapped = (code & 256u) != 0;   // ranks go through the general body: the branch-free one is built on the subtraction
-        const bool full_block = N == kBlockElems && d->real == kBlockElems && expect <= cap && simple_sub && !mapped;
+        // ranks go through the general body: the branch-free one is built on the subtraction
+        const bool full_block = !MAPPED && N == kBlockElems && d->real == kBlockElems && expect <= cap && simple_sub;
         // preparation: ranks of the wide groups and expanded records
         if (hbits > 0) {
             // the branch-free body wants narrow groups to point at the flip slot and flipped records
@@ -909,17 +909,15 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             r.out = d->out;
             r.high = d->high;
             r.lo = d->lo;
-            if (mapped) {
-                r.n = 0;
-                r.c4 = st + kStageRankTable;
-            }
+            if constexpr (MAPPED) r.c4 = st + kStageRankTable;  // the ranked bodies' table
             r.real = d->real;
         }
         if (consumer_barrier_or(*abort_flag != 0)) break;
-        switch (code & 255u) {
+        switch (code) {
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
-        if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid);     \
+        if constexpr (MAPPED) decode_block<DTV, MV, HV, true>(r, st + o_low, st + o_smhi, N, tid); \
+        else if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid); \
         else decode_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, N, tid);                  \
         break;
             ENEC_FOR_EACH_MH(ENEC_CASE, DT)
@@ -927,7 +925,8 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
         if constexpr (DTV != ENEC_FP16) {                                                    \
-            if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid); \
+            if constexpr (MAPPED) decode_block<DTV, MV, HV, true>(r, st + o_low, st + o_smhi, N, tid); \
+            else if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid); \
             else decode_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, N, tid);              \
         }                                                                                    \
         break;

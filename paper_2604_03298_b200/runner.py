@@ -125,15 +125,16 @@ class CodecSet:
         if st != 0:
             raise enec.EnecError(st, f"enec_compress tensor {i}")
 
-    def decompress_all(self, n_streams: int = 1) -> None:
+    def decompress_all(self, n_streams: int = 1, ranked: bool = False) -> None:
         """One enec_decompress per tensor, on the current stream or spread over n_streams side streams. The
         stream length passed is the buffer's capacity; the true length is in the stream header and is checked
         against it on the device."""
-        self.spread(n_streams, self._decompress_one)
+        self.spread(n_streams, lambda i: self._decompress_one(i, ranked))
 
-    def _decompress_one(self, i: int) -> None:
+    def _decompress_one(self, i: int, ranked: bool = False) -> None:
         t = self.raw[i]
-        st = enec.enec_decompress(self.streams[i], self.streams[i].numel(), _DT[t.dtype], t.numel(),
+        fn = enec.enec_decompress_ranked if ranked else enec.enec_decompress
+        st = fn(self.streams[i], self.streams[i].numel(), _DT[t.dtype], t.numel(),
                                   self.outs[i], self.status)
         if st != 0:
             raise enec.EnecError(st, f"enec_decompress tensor {i}")
