@@ -135,7 +135,7 @@ __host__ __device__ inline int width_eq1(int b, int l, int h, int E) {
 
 // Eq. 4 at L = 16 for every m in 1..n, given the number of elements per bit width of the stored value; one
 // thread. Plain IEEE double, one rounding per operation, no fused multiply-add; ties go to the smaller m.
-__device__ inline int choose_m(const unsigned long long* width_count, int n) {
+__device__ __forceinline__ int choose_m(const unsigned long long (&width_count)[9], int n) {
     unsigned long long total = 0;
     for (int w = 0; w <= 8; ++w) total += width_count[w];
     unsigned long long cnt = width_count[0];
