@@ -8,6 +8,7 @@
 
 #include "enec_decode.cuh"
 #include "enec_encode.cuh"
+#include "enec_launch.cuh"
 
 namespace enec {
 
@@ -15,7 +16,6 @@ std::atomic<uint64_t> g_launches{0};
 
 struct DeviceInfo {
     int sms = 0;
-    bool decode_attr_set[3] = {false, false, false};
     bool hist_attr_set[3] = {false, false, false};
     bool encode_attr_set[3] = {false, false, false};
     bool batch_attr_set[3] = {false, false, false};
@@ -30,48 +30,7 @@ static DeviceInfo& device_info(int dev) {
     return d;
 }
 
-// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
-// stream drains; it waits for the predecessor's completion itself (pdl_wait) before touching memory.
-template <class... KernelArgs, class... Args>
-static cudaError_t launch_pdl(void (*kernel)(KernelArgs...), uint32_t grid, uint32_t threads, size_t smem,
-                              cudaStream_t stream, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(threads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, KernelArgs(args)...);
-}
-
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
-
-template <int DT>
-static enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked = false) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
-    DeviceInfo& info = device_info(dev);
-    if (!info.decode_attr_set[DT]) {
-        if (cudaFuncSetAttribute(enec_decode_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 int(kDecodeSmemBytes)) != cudaSuccess ||
-            cudaFuncSetAttribute(enec_decode_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 int(kDecodeSmemBytes)) != cudaSuccess)
-            return ENEC_ERR_CUDA;
-        info.decode_attr_set[DT] = true;
-    }
-    uint32_t grid = uint32_t(info.sms) * 3;  // three resident CTAs per SM
-    if (grid > batch.total_blocks) grid = batch.total_blocks;
-    if (grid == 0) grid = 1;
-    const cudaError_t err =
-        ranked ? launch_pdl(enec_decode_kernel<DT, true>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status)
-               : launch_pdl(enec_decode_kernel<DT, false>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
-}
 
 // Device scratch, one area per (device, stream, purpose): for the compressor control words and one state
 // word per block, for a batched call the tensor descriptors. Grown when a larger request arrives;
@@ -321,9 +280,7 @@ static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype d
                                      uint64_t(in_size)};
     batch.inline_prefix[0] = 0;
     batch.inline_prefix[1] = batch.total_blocks;
-    return dt == ENEC_BF16   ? launch_decode<ENEC_BF16>(batch, d_status, stream, ranked)
-           : dt == ENEC_FP16 ? launch_decode<ENEC_FP16>(batch, d_status, stream, ranked)
-                             : launch_decode<ENEC_FP32>(batch, d_status, stream, ranked);
+    return launch_decode_any(dt, batch, d_status, stream, ranked);
 }
 
 enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
@@ -383,9 +340,7 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
         batch.jobs = reinterpret_cast<const DecodeJob*>(scratch);
         batch.prefix = reinterpret_cast<const uint32_t*>(scratch + jobs_bytes);
     }
-    return dt == ENEC_BF16   ? launch_decode<ENEC_BF16>(batch, d_status, stream)
-           : dt == ENEC_FP16 ? launch_decode<ENEC_FP16>(batch, d_status, stream)
-                             : launch_decode<ENEC_FP32>(batch, d_status, stream);
+    return launch_decode_any(dt, batch, d_status, stream, false);
 }
 
 enec_status enec_compress(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,

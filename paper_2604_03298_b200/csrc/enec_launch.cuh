@@ -1,0 +1,36 @@
+// Host-side launch helpers shared by the library's translation units.
+#pragma once
+
+#include <atomic>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "enec.h"
+
+namespace enec {
+
+extern std::atomic<uint64_t> g_launches;  // kernels launched by the library (enec_launch_count)
+
+struct DecodeBatch;
+// Launches the decode kernel instance for dt (and for the frequency-rank variant when ranked) over `batch`.
+enec_status launch_decode_any(int dt, const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked);
+
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
+// stream drains; it waits for the predecessor's completion itself (pdl_wait) before touching memory.
+template <class... KernelArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KernelArgs...), uint32_t grid, uint32_t threads, size_t smem,
+                              cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KernelArgs(args)...);
+}
+
+}  // namespace enec
