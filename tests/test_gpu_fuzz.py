@@ -95,3 +95,30 @@ def test_batched_calls(oracle, seed):
             got = bufs[i][:nbytes[i]].cpu().numpy()
             assert got.size == want.size and np.array_equal(got, want), (seed, case, i, counts[i])
             assert np.array_equal(from_dev(outs[i], dt, w), w), (seed, case, i, counts[i])
+
+
+@pytest.mark.parametrize("seed", [31, 32])
+def test_ranked_calls(oracle, seed):
+    """The frequency-rank variant over the same random inputs."""
+    import paper_2604_03298_b200 as enec
+    rng = np.random.default_rng(seed)
+    for case in range(80):
+        dt = int(rng.integers(0, 3))
+        count = max(0, int(rng.choice([rng.integers(0, 200), rng.integers(0, 40000), rng.integers(0, 400000),
+                                       16384 * int(rng.integers(1, 20)) + int(rng.integers(-2, 3))])))
+        w = draw(rng, dt, count)
+        want = oracle.compress_ranked(w, dt)
+        cap = enec.enec_max_compressed_size_ranked(dt, count)
+        buf = torch.full((cap + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+        size = torch.zeros(1, dtype=torch.int64, device="cuda")
+        status = status_tensor()
+        assert enec.enec_compress_ranked(to_dev(w, dt), dt, count, buf, cap, size, status) == 0
+        out = torch.empty(count + 16, dtype=TD[dt], device="cuda")
+        d_want = torch.from_numpy(want).cuda()
+        assert enec.enec_decompress_ranked(d_want, d_want.numel(), dt, count, out, status) == 0
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, (seed, case, dt, count)
+        got = buf[:int(size.item())].cpu().numpy()
+        assert got.size == want.size and np.array_equal(got, want), (seed, case, dt, count)
+        assert (buf[cap:] == 0xA5).all()
+        assert np.array_equal(from_dev(out[:count], dt, w), w), (seed, case, dt, count)
