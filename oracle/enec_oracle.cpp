@@ -13,6 +13,7 @@
 
 #include <cstring>
 #include <algorithm>
+#include <utility>
 #include <vector>
 
 namespace {
@@ -100,44 +101,41 @@ uint32_t get_u32(const uint8_t* p) { uint32_t v = 0; for (int i = 0; i < 4; ++i)
 uint64_t get_u64(const uint8_t* p) { uint64_t v = 0; for (int i = 0; i < 8; ++i) v |= uint64_t(p[i]) << (8 * i); return v; }
 
 // ---- Algorithm 2, hierarchical halving bit-packing with byte normalisation ----------------------
-// `data` is taken by value: the algorithm overwrites its lanes.
-std::vector<uint8_t> alg2_pack(std::vector<uint16_t> data, int a) {
-    size_t total_length = 0;
-    int width = a;
-    size_t length = data.size();
-    std::vector<uint8_t> normalized_bytes;
+// Written as the recursion the text describes: a sub-block of lanes, each carrying `bits` payload bits, is
+// folded (the upper half of the lanes moves above the payload of the lower half) until a lane holds at least a
+// byte or one lane is left; the low byte of every lane is stored; whatever is above the byte forms the next
+// sub-block, which goes through the same procedure.
+void normalise_sub_block(std::vector<uint16_t> lanes, int bits, std::vector<uint8_t>& stored) {
+    if (bits <= 0) return;
+    while (lanes.size() > 1 && bits < 8) {
+        const size_t keep = lanes.size() / 2;
+        for (size_t lane = 0; lane < keep; ++lane)
+            lanes[lane] = uint16_t(lanes[lane] | (lanes[keep + lane] << bits));
+        lanes.resize(keep);
+        bits *= 2;
+    }
+    std::vector<uint16_t> overflow;
+    overflow.reserve(lanes.size());
+    for (uint16_t v : lanes) {
+        stored.push_back(uint8_t(v & 0xFF));
+        overflow.push_back(uint16_t(v >> 8));
+    }
+    normalise_sub_block(std::move(overflow), bits - 8, stored);
+}
 
-    while (width > 0) {
-        // hierarchical halving: merge the upper half into the lower half until a byte is filled
-        while (length > 1 && width < 8) {
-            length = length / 2;
-            for (size_t i = 0; i < length; ++i)
-                data[i] = uint16_t(data[i] | (data[i + length] << width));
-            width = width * 2;
-        }
-        // byte normalisation: peel the low byte of every lane, keep the overflow in the lane
-        for (size_t j = 0; j < length; ++j) {
-            normalized_bytes.push_back(uint8_t(data[j] & 0xFF));
-            data[j] = uint16_t(data[j] >> 8);
-        }
-        width = width - 8;
-        total_length = total_length + length;
-    }
-    // pad to an even number of bytes
-    if (total_length % 2 != 0) {
-        normalized_bytes.push_back(0);
-        total_length = total_length + 1;
-    }
-    // final fold: 16-bit word i = byte i | byte (i + half) << 8, written little-endian
-    std::vector<uint8_t> byte_stream;
-    byte_stream.reserve(total_length);
-    size_t half = total_length / 2;
+std::vector<uint8_t> alg2_pack(const std::vector<uint16_t>& values, int a) {
+    std::vector<uint8_t> stored;
+    normalise_sub_block(values, a, stored);
+    if (stored.size() % 2 != 0) stored.push_back(0);  // an even number of bytes: whole 16-bit words
+    // last pass: 16-bit word i takes byte i as its low byte and byte i + half as its high byte; words are
+    // written little-endian
+    const size_t half = stored.size() / 2;
+    std::vector<uint8_t> stream(stored.size());
     for (size_t i = 0; i < half; ++i) {
-        uint16_t output_data = uint16_t(normalized_bytes[i] | (normalized_bytes[i + half] << 8));
-        byte_stream.push_back(uint8_t(output_data & 0xFF));
-        byte_stream.push_back(uint8_t(output_data >> 8));
+        stream[2 * i] = stored[i];
+        stream[2 * i + 1] = stored[half + i];
     }
-    return byte_stream;
+    return stream;
 }
 
 // Inverse of Algorithm 2: replay the forward schedule of folds and byte extractions, then undo the

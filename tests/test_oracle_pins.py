@@ -273,7 +273,8 @@ def _check_stream(oracle, fx):
     words = np.array([int(t, 16) for t in fx["words"][0].split()], dtype=np.uint16)
     assert words.size == count
     params = tuple(map(int, fx["params"][0].split())) if "params" in fx else None
-    expect = np.concatenate([hexbytes(fx[k][0]) for k in ("header", "table", "mask", "low", "sm", "high")])
+    keys = ("header", "table", "mask", "low", "smhi", "sm", "high") if dt == 1 else ("header", "table", "mask", "low", "sm", "high")
+    expect = np.concatenate([hexbytes(fx[k][0]) for k in keys])
     assert hexbytes(fx["header"][0]).size == 64
     got = oracle.compress(words, dt, params)
     assert got.tolist() == expect.tolist()
@@ -286,6 +287,85 @@ def test_stream_hand_16(oracle):
 
 def test_stream_hand_32(oracle):
     _check_stream(oracle, read_fixture("stream_hand_32.txt"))
+
+
+def test_stream_hand_fp16(oracle):
+    # fixes, byte by byte, the 3-bit sign/mantissa-high plane: its width, its bit order (sign above mantissa bits
+    # 9..8), its Algorithm 2 packing and its place between the low plane and the byte plane
+    fx = read_fixture("stream_hand_fp16.txt")
+    assert int(fx["dtype"][0]) == 1
+    _check_stream(oracle, fx)
+
+
+def test_fp16_plane_position_and_content_on_a_large_tensor(oracle):
+    # independent of the hand trace: the section after the low plane, undone with the a = 3 closed form of
+    # Algorithm 2 for a full block (numpy, not the oracle's unpacker), is sign<<2 | mantissa[9:8] of every element
+    rng = np.random.default_rng(41)
+    count = 2 * 16384
+    words = rng.integers(0, 1 << 16, count).astype(np.uint16)
+    s = oracle.compress(words, 1, (15, 5, 2))
+    a16 = lambda v: (v + 15) // 16 * 16
+    off = 64 + a16(4 * 3) + a16(2048 // 8) + a16(count * 2 // 8)
+    want = (((words >> 15) << 2) | ((words >> 8) & 3)).astype(np.uint32)
+    for k in range(2):
+        sec = s[off + k * 6144: off + (k + 1) * 6144]
+        nb = np.concatenate([sec[0::2], sec[1::2]]).astype(np.uint32)        # undo the final fold
+        r = np.concatenate([nb[4096:] & 15, nb[4096:] >> 4])                 # residue nibbles of lanes 0..4095
+        lane = nb[:4096] | (r << 8)
+        e = np.concatenate([lane & 7, (lane >> 6) & 7, (lane >> 3) & 7, (lane >> 9) & 7])
+        assert e.tolist() == want[k * 16384:(k + 1) * 16384].tolist()
+    byte_plane = s[off + 2 * 6144: off + 2 * 6144 + count]
+    assert byte_plane.tolist() == (words & 0xFF).tolist()
+
+
+def test_fp16_gaussian_lands_on_table5_and_table4(oracle):
+    # Table 5: the fp16 models use (7, 4, 3, 16) and (11, 5, 3, 16); Table 4: ratios 1.12 and 1.09. Gaussian fp16
+    # weights at checkpoint scales must land in the same regime: n <= E = 5, m = 3, b a little above the mode.
+    fx = read_fixture("table5_params.txt")
+    rows = [tuple(map(int, fx[k][0].split())) for k in ("Mistral-fp16", "Diffusion-fp16")]
+    assert {r[2:] for r in rows} == {(3, 16)} and {r[1] for r in rows} == {4, 5}
+    t4 = read_fixture("table4_ratios.txt")
+    ratios = [float(t4[k][0]) for k in ("Mistral-fp16", "Diffusion-fp16")]
+    lo, hi = min(ratios) - 0.02, max(ratios) + 0.02
+    import torch
+    for std, seed in ((0.02, 0), (0.01, 1), (0.05, 2)):
+        g = torch.Generator().manual_seed(seed)
+        w = (torch.randn(1 << 21, generator=g) * std).to(torch.float16).view(torch.int16).numpy().view(np.uint16)
+        s = oracle.compress(w, 1)
+        b, n, m = int(s[20]), int(s[21]), int(s[22])
+        assert n in (4, 5) and m == 3 and min(r[0] for r in rows) <= b <= max(r[0] for r in rows) + 1, (std, b, n, m)
+        assert lo < w.nbytes / s.size < hi, (std, w.nbytes / s.size)
+        # the sign/mantissa bits cost exactly 11 per element (8 + 3): what is left is Eq. 4's exponent cost
+        A = int(s[32:36].view(np.uint32)[0])
+        exp_bits = (w.size / 16 + w.size * m + 16 * (n - m) * A) / w.size
+        assert abs(8 * s.size / w.size - (11 + exp_bits)) < 0.01
+
+
+def _sizes_case(oracle, row, dt):
+    count, n, m, A, nblocks, padded, groups, total = map(int, row.split())
+    b, wide_x, shift = (123, 125, 7) if dt == 0 else (10, 11, 10)
+    x = np.full(count, b, np.uint16)
+    flagged = np.arange(A) * 16               # one wide value in each of the first A groups
+    flagged = flagged[flagged < count]
+    assert flagged.size == A
+    x[flagged] = wide_x
+    words = (x << shift).astype(np.uint16)
+    s = oracle.compress(words, dt, (b, n, m))
+    assert s.size == total
+    hdr = s[:64]
+    assert int(hdr[24:28].view(np.uint32)[0]) == nblocks
+    assert int(hdr[28:32].view(np.uint32)[0]) == groups
+    assert int(hdr[32:36].view(np.uint32)[0]) == A
+    assert int(hdr[40:48].view(np.uint64)[0]) == total
+    assert oracle.max_compressed_size(dt, count) >= total
+    assert np.array_equal(oracle.decompress(s, dt, count), words)
+
+
+def test_sizes_closed_form_fp16(oracle):
+    fx = read_fixture("sizes_hand.txt")
+    assert len(fx["case_fp16"]) == 5
+    for row in fx["case_fp16"]:
+        _sizes_case(oracle, row, 1)
 
 
 def test_sizes_closed_form(oracle):
