@@ -43,6 +43,53 @@ def dtype_code(dtype):
     return {"torch.bfloat16": 0, "torch.float16": 1, "torch.float32": 2}[str(dtype)]
 
 
+def decode_traffic_per_element():
+    """dram__bytes_read.sum + dram__bytes_write.sum of enec_decode_kernel per element, from the counters of the
+    last ncu capture (a small text file kept beside the capture's summary), or None when the kernel's source has
+    changed since the capture was taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "decode_kernel_dram_counters.txt")
+    try:
+        rec = dict(line.split(":", 1) for line in open(path) if ":" in line and not line.startswith("#"))
+        rec = {k.strip(): v.strip() for k, v in rec.items()}
+        h = hashlib.sha256()
+        for name in rec["source_files"].split():
+            h.update(open(os.path.join(ROOT, "paper_2604_03298_b200", "csrc", name), "rb").read())
+        if h.hexdigest() != rec["source_sha256"]:
+            return None, "the decode kernel's source has changed since the ncu capture"
+        per_elem = (float(rec["dram_bytes_read"]) + float(rec["dram_bytes_write"])) / float(rec["elements"])
+        return per_elem, f"scaled per element from the ncu capture of {rec['workload']}"
+    except Exception as e:   # no file, or not readable: no figure
+        return None, f"no counters on file ({type(e).__name__})"
+
+
+def launch_ranks(n, argv):
+    """Starts this script again as n ranks on this node (torch.distributed.run, one process per GPU) and returns
+    their exit code. The ranks find RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* in their environment."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
+def run_spawn_selftest(args):
+    """The host logic of an N-rank run without any GPU: rendezvous (gloo), max / sum over ranks, one line from
+    rank 0. Used by the CPU tests of the launch path."""
+    import torch.distributed as dist
+    from paper_2604_03298_b200 import runner
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    dist.init_process_group("gloo")
+    slowest = runner.max_over_ranks(10.0 + rank)
+    total = runner.sum_over_ranks(100.0)
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps({"spawn_selftest": True, "n_gpus": world, "max_over_ranks": slowest, "sum_over_ranks": total}))
+    dist.destroy_process_group()
+
+
 def measured_peak_gbs():
     """HBM copy bandwidth measured on this machine (generated file), else the stated fallback."""
     try:
@@ -242,6 +289,9 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    if world != args.gpus:
+        raise RuntimeError(f"--gpus {args.gpus} but {world} rank(s) are running: start it as `python bench.py --gpus N` "
+                           "or under torch.distributed.run with --nproc-per-node N")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -318,8 +368,17 @@ def run_ours(args):
     total_launches = int(runner.sum_over_ranks(launches))
 
     # end to end through host buffers (pinned): host stream -> device -> decompress -> host tensor, and the
-    # compress direction likewise, on one decoder layer of this rank's set
-    layer = [i for i, s in enumerate(specs) if s.name.startswith("l0.")][:9] or list(range(min(9, len(specs))))
+    # compress direction likewise, on a sample of this rank's set: its first tensors up to about 2 GB of raw bytes
+    # (the link, not the codec, bounds this number, and pinning the whole set would take tens of GB of host memory)
+    layer, e2e_budget = [], 2.2e9
+    for i, t in enumerate(cs.raw):
+        if specs[i].numel * t.element_size() > 600e6:
+            continue   # the embedding alone would be the whole sample
+        layer.append(i)
+        e2e_budget -= specs[i].numel * t.element_size()
+        if e2e_budget <= 0:
+            break
+    e2e_steps = max(1, min(args.steps, 5))
     h_streams = [torch.empty(int(cs.sizes[i].item()), dtype=torch.uint8).pin_memory() for i in layer]
     h_raw = [torch.empty(cs.raw[i].numel(), dtype=cs.raw[i].dtype).pin_memory() for i in layer]
     for h, i in zip(h_streams, layer):
@@ -354,17 +413,18 @@ def run_ours(args):
     def e2e_compress():
         cs.spread(args.spread_streams, e2e_compress_one, len(layer))
 
-    def time_e2e(fn):
+    def time_e2e(fn, steps=None):
+        steps = steps or args.steps
         for _ in range(2):
             fn()
         barrier()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for _ in range(args.steps):
+        for _ in range(steps):
             fn()
         b.record()
         barrier()
-        return runner.max_over_ranks(a.elapsed_time(b) / args.steps)
+        return runner.max_over_ranks(a.elapsed_time(b) / steps)
 
     # the same decompress pass as one batched launch (not part of `value`: the workload says tensor by tensor)
 
@@ -414,11 +474,32 @@ def run_ours(args):
     cs.check_status()
     cs.verify_roundtrip()
 
-    ms_e2e_dec = time_e2e(e2e_decompress)
-    ms_e2e_comp = time_e2e(e2e_compress)
+    ms_e2e_dec = time_e2e(e2e_decompress, e2e_steps)
+    ms_e2e_comp = time_e2e(e2e_compress, e2e_steps)
     cs.check_status()
     for h, i in zip(h_raw, layer):  # the host copy of the last decompress must be the tensor
         assert (host_words(h) == host_words(cs.raw[i])).all()
+
+    # side number: the ratio when the normal generator's rare exact zeros are left in (one zero sets the lowest
+    # occupied exponent of its tensor to 0 and with it n = 8): the largest tensor of the set and the sample's tensors
+    zeros_kept = None
+    if rank == 0 and cfg in (1, 2, 3):
+        biggest = max(range(len(specs)), key=lambda i: specs[i].numel)
+        zr = zc = zeros = 0
+        for i in sorted(set([biggest] + layer[:9])):
+            t = synth.make_tensor(specs[i], "cuda", keep_zeros=True)
+            zeros += int((t == 0).sum().item())
+            st = enec.enec_compress(t, dtype_code(t.dtype), t.numel(), cs.streams[i], cs.streams[i].numel(),
+                                    cs.sizes[i:i + 1], cs.status)
+            assert st == 0
+            zr += t.numel() * t.element_size()
+            zc += int(cs.sizes[i].item())
+            del t
+        zeros_kept = {"compression_ratio": zr / zc, "exact_zeros": zeros, "raw_bytes": zr,
+                      "sample": f"{len(set([biggest] + layer[:9]))} tensors: the largest of the set and one decoder layer"}
+        cs.compress_all()
+        torch.cuda.synchronize()
+        cs.check_status()
 
     if rank != 0:
         if world > 1:
@@ -430,14 +511,16 @@ def run_ours(args):
     dec_moved = (raw_bytes + comp_bytes)                       # algorithmic bytes of one decompress pass (this rank)
     achieved = dec_moved / (ms_dec * 1e-3) / 1e9
     elems = sum(t.numel() for t in cs.raw)
-    all_bf16 = all(t.dtype == torch.bfloat16 for t in cs.raw)   # the committed DRAM counters are bf16's
+    all_bf16 = all(t.dtype == torch.bfloat16 for t in cs.raw)   # the DRAM counters on file are bf16's
+    traffic_per_elem, traffic_note = decode_traffic_per_element()
     roofline = {
         "kernel": "enec_decode_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth",
         "algorithmic_bytes_per_launch": dec_moved / n_dec, "launches_per_step": n_dec,
         "avg_launch_us": ms_dec * 1e3 / n_dec,
         "avg_launch_note": "duration of the decompress pass / its launches (launches of different streams overlap)",
-        "traffic": DECODE_DRAM_BYTES_PER_ELEM * elems / n_dec if DECODE_DRAM_BYTES_PER_ELEM and all_bf16 else None,
+        "traffic": traffic_per_elem * elems / n_dec if traffic_per_elem and all_bf16 else None,
+        "traffic_note": traffic_note if all_bf16 else "the counters on file are for bf16 streams",
         "compress": {"achieved": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9,
                      "frac": (raw_bytes + comp_bytes) / (ms_comp * 1e-3) / 1e9 / peak,
                      "note": "algorithmic bytes = read raw once + write stream; the histogram pass reads raw again"},
@@ -454,7 +537,7 @@ def run_ours(args):
         gpu_sizes = [int(cs.sizes[i].item()) for i in sample_idx]
         assert sum(gpu_sizes) == scomp, "GPU and oracle stream sizes differ on the sample"
         cpu = {"value": sraw / td / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-               "sample": f"{len(sample_idx)} tensors of the workload ({sraw / 1e6:.0f} MB raw), single thread",
+               "sample": f"sample: {len(sample_idx)} tensors of the workload ({sraw / 1e6:.0f} MB raw), single thread",
                "compress": {"value": sraw / tc / 1e9, "unit": "GB/s"}, "compression_ratio": sraw / scomp}
         all_dec, all_comp, all_threads = time_oracle_all_cores(words, dtype_code(cs.raw[sample_idx[0]].dtype))
         cpu["all_cores"] = {"value": all_dec, "unit": "GB/s", "cores": all_threads, "compress": {"value": all_comp, "unit": "GB/s"},
@@ -501,6 +584,7 @@ def run_ours(args):
                              "launches_per_pass": 2 * len({t.dtype for t in cs.raw}),
                              "note": "same tensors through enec_compress_batched (one call per dtype of the set)"},
         "compression_ratio": total_raw / total_comp,
+        "compression_ratio_zeros_kept": zeros_kept,
         "ablation_frequency_ranks": {
             "compression_ratio": total_raw / ranked_bytes,
             "decompress": {"value": total_raw / (ms_dec_ranked * 1e-3) / 1e9, "unit": "GB/s"},
@@ -512,9 +596,10 @@ def run_ours(args):
         "cpu_vectorised": cpu_vec,
         "e2e": {"value": e2e_raw * world / (ms_e2e_dec * 1e-3) / 1e9, "unit": "GB/s",
                 "h2d_bytes_per_step": e2e_comp, "d2h_bytes_per_step": e2e_raw,
-                "workload": "one decoder layer of the set, tensor by tensor: pinned host stream -> device -> "
-                            "enec_decompress -> pinned host" + (f", tensors spread over {args.spread_streams} streams"
-                                                                  if args.spread_streams > 1 else ""),
+                "workload": f"sample: the first {len(layer)} tensors of the set without its embedding ({e2e_raw / 1e9:.2f} GB raw), "
+                            "tensor by tensor: pinned host stream -> device -> enec_decompress -> pinned host"
+                            + (f", tensors spread over {args.spread_streams} streams" if args.spread_streams > 1 else ""),
+                "steps": e2e_steps,
                 "compress": {"value": e2e_raw * world / (ms_e2e_comp * 1e-3) / 1e9, "unit": "GB/s",
                              "h2d_bytes_per_step": e2e_raw, "d2h_bytes_per_step": e2e_comp}},
         "gpu_launches": total_launches,
@@ -524,13 +609,6 @@ def run_ours(args):
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
-
-
-# dram__bytes_read.sum + dram__bytes_write.sum per element of enec_decode_kernel from the committed ncu capture
-# (profiles/decode_kernel_llama_layer.md: 85.54 MB read + 62.36 MB written for the 58,720,256 elements of
-# gate_proj). Below the algorithmic 3.475 B/element because part of the output is still dirty in L2 when the
-# kernel ends. Set to None when the kernel changes until a new capture exists.
-DECODE_DRAM_BYTES_PER_ELEM = (85.537024e6 + 62.355456e6) / 58720256
 
 
 def main():
@@ -546,9 +624,24 @@ def main():
     ap.add_argument("--spread-streams", type=int, default=8,
                     help="streams of the extra multi-stream measurement and of the end-to-end pass")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--spawn-selftest", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.gpus > 1 and "RANK" not in os.environ:
+        # started by hand for several GPUs: become the launcher of N ranks, one per GPU
+        if not args.spawn_selftest:
+            import torch
+            have = torch.cuda.device_count()
+            if have < args.gpus:
+                print(f"bench.py: --gpus {args.gpus} needs {args.gpus} CUDA devices, {have} visible", file=sys.stderr)
+                sys.exit(2)
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
+    if args.spawn_selftest:
+        run_spawn_selftest(args)
     else:
         run_ours(args)
 

@@ -105,7 +105,7 @@ template <int DT>
 static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool search, int* d_status, DeviceInfo& info,
                                  cudaStream_t stream) {
     if (search) {
-        const uint32_t smem = HistShape<DT>::kWarpBytes * (kHistThreads / 32);
+        const uint32_t smem = HistShape<DT>::kBytes;
         if (!info.hist_attr_set[DT]) {
             if (cudaFuncSetAttribute(enec_histogram_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      int(smem)) != cudaSuccess ||
@@ -150,7 +150,7 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
 template <int DT>
 static enec_status launch_encode_batched(const EncodeJob* d_jobs, const HistUnit* d_units, uint32_t n_units,
                                          const EncodeBatch& batch, int* d_status, DeviceInfo& info, cudaStream_t stream) {
-    const uint32_t hist_smem = HistShape<DT>::kWarpBytes * (kHistThreads / 32);
+    const uint32_t hist_smem = HistShape<DT>::kBytes;
     if (!info.batch_attr_set[DT]) {
         if (cudaFuncSetAttribute(enec_histogram_batched_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(hist_smem)) != cudaSuccess ||

@@ -585,24 +585,6 @@ static_assert(sizeof(DecodeShared) == 128, "control area is 128 bytes");
     X(DT, 7, 0) X(DT, 7, 1)                                                                           \
     X(DT, 8, 0)
 
-// Bounded wait of any number of threads: each try suspends the thread for up to 20 us or until the phase
-// completes, and there are at most 2^16 tries (about a second); also gives up when the CTA aborts.
-__device__ __forceinline__ bool suspended_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < (1u << 16); ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
-            : "memory");
-        if (ok) return true;
-        if (*abort_flag) return false;
-    }
-    return false;
-}
-
 // What the loader tells the consumers about the block in a stage (first bytes of the stage).
 struct BlockDesc {
     uint32_t first;     // offset of the block's first record inside the staged window

@@ -83,37 +83,40 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p) {
 // ---------------------------------------------------------------------------------------------------
 // Sec. 5.5 phase 1: histogram of the exponent field.
 //
-// Every warp keeps eight copies of the histogram in shared memory (lane l adds to copy l mod 8; a bin's
-// eight 32-bit counters fill one 32-byte row), so the adds of a warp instruction spread over all banks and
-// at most four lanes can meet on a counter. Counting is one `red.shared.add` per value: no read-modify-
-// write chain in the thread, no overflow, nothing to fold until the end.
+// A CTA keeps 32 copies of the histogram in shared memory, one per lane number: bin x is a row of 32 counters
+// (128 bytes) and lane l of every warp adds to counter l of the row, so the 32 adds of a warp instruction go
+// to 32 different banks whatever the values are (weights concentrate in three or four exponents, the worst
+// case for anything shared between lanes), and an instruction is one pass through shared memory. Warps share
+// the rows: the adds are atomic. Counting is one `red.shared.add` per value: no read-modify-write chain in
+// the thread, no overflow, nothing to fold until the end.
 // ---------------------------------------------------------------------------------------------------
 template <int DT>
 struct HistShape {
     static constexpr int E = DT == ENEC_FP16 ? 5 : 8;
     static constexpr int kBins = 1 << E;
     static constexpr int kPerLoad = DT == ENEC_FP32 ? 4 : 8;  // values in a 16-byte load
-    static constexpr int kCopies = 8;                    // copies of the histogram per warp
-    static constexpr int kWarpBytes = kBins * kCopies * 4;
+    static constexpr int kCopies = 32;                   // copies of the histogram per CTA: one per lane number
+    static constexpr int kRowBytes = kCopies * 4;
+    static constexpr int kBytes = kBins * kRowBytes;
 };
 
-// One value counted: a fire-and-forget shared-memory add on the copy of the warp's histogram that the lane
-// uses (eight copies per warp, 32 bytes per bin), addressed straight from the word's bits.
+// One value counted: a fire-and-forget shared-memory add on the lane's counter of the value's row, addressed
+// straight from the word's bits.
 __device__ __forceinline__ void red_add_one(uint32_t addr) {
     asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(addr), "r"(1u) : "memory");
 }
 
 template <int DT>
 __device__ __forceinline__ void count_word_pair(uint32_t base, uint32_t w) {
-    // two 16-bit values per 32-bit word (one fp32 value); bin x sits at byte x * 32 of the warp's area
+    // two 16-bit values per 32-bit word (one fp32 value); bin x sits at byte x * 128 of the CTA's area
     if (DT == ENEC_FP32) {
-        red_add_one(base + ((w >> 18) & 0x1FE0u));   // x = bits 30..23
+        red_add_one(base + ((w >> 16) & 0x7F80u));   // x = bits 30..23
     } else if (DT == ENEC_BF16) {
-        red_add_one(base + ((w >> 2) & 0x1FE0u));    // x = bits 14..7
-        red_add_one(base + ((w >> 18) & 0x1FE0u));
+        red_add_one(base + (w & 0x7F80u));           // x = bits 14..7: already in place
+        red_add_one(base + ((w >> 16) & 0x7F80u));
     } else {
-        red_add_one(base + ((w >> 5) & 0x3E0u));     // x = bits 14..10
-        red_add_one(base + ((w >> 21) & 0x3E0u));
+        red_add_one(base + ((w >> 3) & 0xF80u));     // x = bits 14..10
+        red_add_one(base + ((w >> 19) & 0xF80u));
     }
 }
 
@@ -245,19 +248,32 @@ __device__ void parameter_search_ranked(EncodeControl* ctl) {
     }
 }
 
+// Sum of a row's 32 counters, by the thread that owns the bin (the rows of neighbouring threads are read
+// in rotated order, so that they do not all go to the same banks); CLEAR leaves the row zeroed.
+template <bool CLEAR>
+__device__ __forceinline__ uint32_t fold_hist_row(uint32_t row, uint32_t tid) {
+    uint32_t sum = 0;
+#pragma unroll
+    for (uint32_t q = 0; q < 8; ++q) {
+        const uint32_t at = row + ((q + tid) & 7) * 16;
+        const uint4 v = lds128(at);
+        sum += v.x + v.y + v.z + v.w;
+        if (CLEAR) sts128(at, make_uint4(0, 0, 0, 0));
+    }
+    return sum;
+}
+
 template <int DT, bool RANKED = false>
 __global__ void __launch_bounds__(kHistThreads, 3)
 enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeControl* ctl) {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t cta_hist[256];
     __shared__ int s_last;
-    constexpr int kWarpBytes = HistShape<DT>::kWarpBytes;
     pdl_launch_dependents();
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t warp_base = smem_u32(smem) + warp * kWarpBytes;
-    const uint32_t base = warp_base + (lane & 7) * 4;
-    for (uint32_t i = tid; i < uint32_t(kWarpBytes / 4) * (kHistThreads / 32); i += kHistThreads)
-        reinterpret_cast<uint32_t*>(smem)[i] = 0;
+    const uint32_t base = smem_u32(smem) + lane * 4;
+    for (uint32_t i = tid; i < uint32_t(HistShape<DT>::kBytes / 16); i += kHistThreads)
+        reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
     cta_hist[tid] = 0;
     __syncthreads();
     pdl_wait();  // nothing above touches global memory
@@ -303,15 +319,7 @@ enec_histogram_kernel(const uint16_t* __restrict__ in, uint64_t count, EncodeCon
         first += stride;
     }
     __syncthreads();
-    if (tid < uint32_t(HistShape<DT>::kBins)) {  // fold the warps' copies of bin `tid`
-        uint32_t sum = 0;
-        for (uint32_t wp = 0; wp < kHistThreads / 32; ++wp) {
-            const uint32_t row = smem_u32(smem) + wp * kWarpBytes + tid * 32;
-            const uint4 lo = lds128(row), hi = lds128(row + 16);
-            sum += lo.x + lo.y + lo.z + lo.w + hi.x + hi.y + hi.z + hi.w;
-        }
-        cta_hist[tid] = sum;
-    }
+    if (tid < uint32_t(HistShape<DT>::kBins)) cta_hist[tid] = fold_hist_row<false>(smem_u32(smem) + tid * HistShape<DT>::kRowBytes, tid);
     __syncthreads();
     if (blockIdx.x == 0 && tid == 0) {  // the values behind the last whole 16-byte load
         constexpr int sh = DT == ENEC_BF16 ? 7 : 10;
@@ -350,13 +358,12 @@ enec_histogram_batched_kernel(const EncodeJob* __restrict__ jobs, const HistUnit
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t cta_hist[256];
     __shared__ int s_last;
-    constexpr int kWarpBytes = HistShape<DT>::kWarpBytes;
     constexpr int kPerLoad = HistShape<DT>::kPerLoad;
     pdl_launch_dependents();
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t base = smem_u32(smem) + warp * kWarpBytes + (lane & 7) * 4;
-    for (uint32_t i = tid; i < uint32_t(kWarpBytes / 4) * (kHistThreads / 32); i += kHistThreads)
-        reinterpret_cast<uint32_t*>(smem)[i] = 0;
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
+    const uint32_t base = smem_u32(smem) + lane * 4;
+    for (uint32_t i = tid; i < uint32_t(HistShape<DT>::kBytes / 16); i += kHistThreads)
+        reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
     cta_hist[tid] = 0;
     __syncthreads();
     pdl_wait();  // nothing above touches global memory
@@ -387,17 +394,8 @@ enec_histogram_batched_kernel(const EncodeJob* __restrict__ jobs, const HistUnit
             }
         }
         __syncthreads();
-        if (tid < uint32_t(HistShape<DT>::kBins)) {  // fold the warps' copies of bin `tid` and clear them for the next unit
-            uint32_t sum = 0;
-            for (uint32_t wp = 0; wp < kHistThreads / 32; ++wp) {
-                const uint32_t row = smem_u32(smem) + wp * kWarpBytes + tid * 32;
-                const uint4 lo = lds128(row), hi = lds128(row + 16);
-                sum += lo.x + lo.y + lo.z + lo.w + hi.x + hi.y + hi.z + hi.w;
-                sts128(row, make_uint4(0, 0, 0, 0));
-                sts128(row + 16, make_uint4(0, 0, 0, 0));
-            }
-            cta_hist[tid] = sum;
-        }
+        // fold the row of bin `tid` and clear it for the next unit
+        if (tid < uint32_t(HistShape<DT>::kBins)) cta_hist[tid] = fold_hist_row<true>(smem_u32(smem) + tid * HistShape<DT>::kRowBytes, tid);
         __syncthreads();
         if (tid == 0 && unit.index + 1 == unit.units_of_job) {  // the values behind the last whole 16-byte load
             constexpr int sh = DT == ENEC_BF16 ? 7 : 10;

@@ -105,8 +105,9 @@ def config_specs(cfg: int, scale: int = 1):
     raise ValueError(f"unknown config {cfg}")
 
 
-def make_tensor(spec: TensorSpec, device="cpu") -> torch.Tensor:
-    """Draws the tensor in fp32 on ``device`` and rounds it to the spec's dtype (nearest even; fp32 stays as drawn)."""
+def make_tensor(spec: TensorSpec, device="cpu", keep_zeros: bool = False) -> torch.Tensor:
+    """Draws the tensor in fp32 on ``device`` and rounds it to the spec's dtype (nearest even; fp32 stays as drawn).
+    keep_zeros: leave the normal generator's rare exact zeros in (see below)."""
     gen = torch.Generator(device=device)
     gen.manual_seed(spec.seed)
     n = spec.numel
@@ -114,7 +115,8 @@ def make_tensor(spec: TensorSpec, device="cpu") -> torch.Tensor:
         t = torch.randn(n, generator=gen, device=device, dtype=torch.float32)
         # A float32 normal generator emits exact 0.0 about once per 2^24 draws; a Gaussian has no atom at
         # zero, and one such value would set the lowest occupied exponent to 0 for the whole tensor.
-        t = torch.where(t == 0, torch.full_like(t, 2.0 ** -10), t)
+        if not keep_zeros:
+            t = torch.where(t == 0, torch.full_like(t, 2.0 ** -10), t)
         t = t * spec.std + spec.mean
     elif spec.dist == "laplace":
         u = torch.rand(n, generator=gen, device=device, dtype=torch.float32) - 0.5

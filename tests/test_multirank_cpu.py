@@ -48,3 +48,33 @@ def test_single_process_passthrough():
     from paper_2604_03298_b200 import runner
     assert runner.max_over_ranks(3.5) == 3.5
     assert runner.shard(list(range(7)), 1, 3) == [1, 4]
+
+
+def _bench(*argv):
+    import subprocess
+    env = dict(os.environ)
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT"):
+        env.pop(k, None)
+    env["CUDA_VISIBLE_DEVICES"] = ""      # the launcher must count no device here, GPU machine or not
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *argv], capture_output=True, text=True,
+                          timeout=300, env=env)
+
+
+def test_bench_gpus_n_refuses_to_pretend():
+    """`bench.py --gpus N` with fewer than N devices exits non-zero with a message; it never prints a line."""
+    r = _bench("--gpus", "2")
+    assert r.returncode != 0
+    assert "needs 2 CUDA devices" in r.stderr
+    assert r.stdout.strip() == ""
+
+
+def test_bench_gpus_n_starts_n_ranks():
+    """The launcher path of `bench.py --gpus 2`: two ranks rendezvous (gloo, no GPU work), rank 0 prints one
+    line with n_gpus = the ranks that really ran."""
+    import json
+    r = _bench("--gpus", "2", "--spawn-selftest")
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2 and rec["max_over_ranks"] == 11.0 and rec["sum_over_ranks"] == 200.0
