@@ -12,7 +12,8 @@
  * compressed). `count` is always a number of elements.
  *
  * All pointers named d_* are DEVICE pointers, 16-byte aligned, owned by the caller. Every call only
- * enqueues work on `stream` and returns; nothing synchronises with the host. Errors the host can see
+ * enqueues work on `stream` and returns; nothing synchronises with the host. The current device's ordinal
+ * must be below 64 (ENEC_ERR_CUDA otherwise). Errors the host can see
  * (null or misaligned pointers, unknown dtype, count >= 2^36, capacity below enec_max_compressed_size)
  * are returned at once. Errors only the device can see (damaged stream, parameters that are not
  * lossless, a wait that ran out) are written to *d_status if d_status is not NULL: the first error wins,
@@ -23,8 +24,10 @@
  * and control words); it is allocated on the first compress call on that stream and kept until exit.
  * The area carries state from one compress call on the stream to the next (that is what saves clearing it
  * every call), so: compress calls on ONE stream are issued by one host thread at a time, and
- * enec_compress / enec_compress_with_params on a stream that is being captured into a CUDA graph return
- * ENEC_ERR_INVALID_ARG (a replay would not see the state). Decompression keeps no state and can be captured.
+ * enec_compress / enec_compress_with_params / enec_compress_batched on a stream that is being captured into a
+ * CUDA graph return ENEC_ERR_INVALID_ARG (a replay would not see the state). Decompression keeps no state and
+ * can be captured; a batched call of more than 16 tensors is then recorded as one launch per 16 tensors, since
+ * a longer list would have to pass through host and scratch memory that a replay cannot rely on.
  */
 #ifndef ENEC_H
 #define ENEC_H
@@ -63,7 +66,7 @@ typedef struct CUstream_st* enec_stream_t;
 size_t enec_max_compressed_size(enec_dtype dt, size_t count);
 
 /*
- * Compress `count` 16-bit values at d_in into d_out (Sec. 5.1 compression flow: split, histogram and
+ * Compress `count` elements of type `dt` at d_in into d_out (Sec. 5.1 compression flow: split, histogram and
  * parameter choice of Sec. 5.5, transform of Sec. 5.3, group widths of Sec. 5.2, Algorithm 2 packing,
  * block-offset prefix sum). out_capacity must be at least enec_max_compressed_size(dt, count).
  * d_out_size (device, 8-byte aligned, may be NULL) receives the stream length, which is also in the
@@ -83,7 +86,7 @@ enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t co
                                       enec_stream_t stream);
 
 /*
- * Decompress the stream at d_in (in_size bytes) into `count` 16-bit values at d_out (Sec. 5.1
+ * Decompress the stream at d_in (in_size bytes) into `count` elements of type `dt` at d_out (Sec. 5.1
  * decompression flow: mask -> prefix sums -> unpack low and high parts -> inverse transform -> rejoin
  * with sign/mantissa). dt and count must match the stream header, else ENEC_ERR_BAD_STREAM is reported in
  * *d_status. The result is bit-identical to the tensor that was compressed.
@@ -119,9 +122,10 @@ typedef struct {
 
 /*
  * Decompress n_items streams of one dtype with a single launch (one entry per tensor, in HOST memory;
- * the call copies the descriptors to the device on `stream`). Meant for checkpoints made of many small
- * tensors, where one launch per tensor would be launch-bound. Same per-tensor semantics as
- * enec_decompress; *d_status holds the first error of any tensor.
+ * the call copies the descriptors to the device on `stream`; the paper's interface has no batch, and host
+ * arrays spare the caller a device copy of its own). Meant for checkpoints made of many small tensors, where
+ * one launch per tensor would be launch-bound. Same per-tensor semantics as enec_decompress, for tensors
+ * without elements too (their 80-byte streams are checked); *d_status holds the first error of any tensor.
  */
 enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items, enec_dtype dt, int* d_status,
                                     enec_stream_t stream);
@@ -148,8 +152,9 @@ enec_status enec_compress_batched(const enec_batch_item* h_items, int n_items, e
  * cudaMalloc would stall other streams (it synchronises the device), and services that have handed the
  * whole device budget to something else. For them this entry point takes its working memory from a
  * fixed array inside the library image (ENEC_NOALLOC_SCRATCH_BYTES, about 0.5 MB, present on every GPU
- * that loads the library for as long as the process lives) and calls neither cudaMalloc nor cudaFree
- * nor any routine that allocates.
+ * that loads the library for as long as the process lives) and makes no cudaMalloc or cudaFree call of its
+ * own, nor a call of a library routine that allocates (what the driver does when it first loads a kernel's
+ * code is outside the library's hands); enec_allocation_count() lets a caller check.
  *
  * Same arguments, stream format and output as enec_compress (the two write identical bytes). Limits and
  * rules that differ:
@@ -168,6 +173,9 @@ enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count,
 
 /* Number of kernels the library has launched in this process (all entry points, all streams). */
 uint64_t enec_launch_count(void);
+
+/* Number of cudaMalloc calls the library has made in this process (scratch areas; never freed before exit). */
+uint64_t enec_allocation_count(void);
 
 /* Library version: 10000 * major + 100 * minor + patch. */
 int enec_version(void);

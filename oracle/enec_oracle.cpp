@@ -8,6 +8,10 @@
  * boundary and is zero padded):
  *   header 64 B | table u32[nblocks+1] | mask | low plane | (fp16: sm-hi plane) | sm plane |
  *   (fp32: sm-lo plane, mantissa bits 15..0, two bytes per element) | high records
+ * Block-wise variant (header byte 7 = 2; Sec. 5.5 run on every block's own histogram): the table is replaced
+ * by a block table of 16-byte entries {b, n, m, 0, u32 sum of m over the blocks before, u64 record bytes before},
+ * nblocks + 1 of them (the last holds the totals); block k's low plane starts at 2048 x (sum of m before it)
+ * and its records at (record bytes before it); header bytes 20..22 are zero.
  */
 #include "enec_oracle.h"
 
@@ -90,6 +94,21 @@ Sections sections(int dtype, size_t count, const Geometry& g, int n, int m, uint
     s.smlo = s.sm + align16(count);
     s.high = s.smlo + (dtype == 2 ? align16(count * 2) : 0);
     s.total = s.high + align16(size_t(a_total) * 2 * (n - m));
+    return s;
+}
+
+// Section offsets of the block-wise variant: low_bytes and high_bytes are the sums over the blocks.
+Sections sections_blockwise(int dtype, size_t count, const Geometry& g, uint64_t low_bytes, uint64_t high_bytes) {
+    Sections s;
+    s.unmap = kHeaderBytes;
+    s.table = kHeaderBytes;
+    s.mask = s.table + align16(16 * (size_t(g.nblocks) + 1));
+    s.low = s.mask + align16((size_t(g.total_groups) + 7) / 8);
+    s.smhi = s.low + align16(size_t(low_bytes));
+    s.sm = s.smhi + (dtype == 1 ? align16(size_t(g.padded_count) * 3 / 8) : 0);
+    s.smlo = s.sm + align16(count);
+    s.high = s.smlo + (dtype == 2 ? align16(count * 2) : 0);
+    s.total = s.high + align16(size_t(high_bytes));
     return s;
 }
 
@@ -312,7 +331,7 @@ uint32_t load_word(const void* in, int dtype, size_t i) {
 }
 
 int encode(const void* in, int dtype, size_t count, bool have_params, int b, int n, int m,
-           uint8_t* out, size_t capacity, size_t* out_size, bool ranked = false) {
+           uint8_t* out, size_t capacity, size_t* out_size, bool ranked = false, bool blockwise = false) {
     if (!known_dtype(dtype)) return ERR_UNSUPPORTED_DTYPE;
     if ((!in && count) || !out || !out_size || (count >> 36)) return ERR_INVALID_ARG;
     const int E = exp_bits(dtype);
@@ -329,7 +348,10 @@ int encode(const void* in, int dtype, size_t count, bool have_params, int b, int
         hist[xe] += 1;
     }
     uint8_t rank_of[256], unmap[256];
-    if (ranked) {
+    if (blockwise) {
+        if (have_params || ranked) return ERR_INVALID_ARG;
+        b = 0; n = 1; m = 1;  // every block chooses its own below
+    } else if (ranked) {
         if (have_params) return ERR_INVALID_ARG;
         rank_mapping(hist.data(), E, rank_of, unmap, &n, &m);
         b = 0;
@@ -346,12 +368,26 @@ int encode(const void* in, int dtype, size_t count, bool have_params, int b, int
     std::vector<uint32_t> table(size_t(g.nblocks) + 1, 0);
     std::vector<uint8_t> mask((size_t(g.total_groups) + 7) / 8, 0);
     std::vector<uint8_t> low, smhi, high;
-    const uint16_t low_mask = uint16_t((1u << m) - 1);
+    uint16_t low_mask = uint16_t((1u << m) - 1);
     uint32_t a_total = 0;
+    std::vector<uint8_t> block_table(blockwise ? 16 * (size_t(g.nblocks) + 1) : 0, 0);
+    uint32_t m_before = 0;
     for (uint32_t k = 0; k < g.nblocks; ++k) {
         size_t first = size_t(k) * kBlock;
         uint32_t real = (k + 1 == g.nblocks) ? g.tail_real : kBlock;
         uint32_t np = (k + 1 == g.nblocks) ? g.tail_padded : kBlock;
+        if (blockwise) {
+            // Sec. 5.5 on the histogram of this block's own (real) elements
+            std::vector<uint64_t> block_hist(size_t(1) << E, 0);
+            for (uint32_t i = 0; i < real; ++i) block_hist[x[first + i]] += 1;
+            param_search(block_hist.data(), E, &b, &n, &m, nullptr, nullptr);
+            low_mask = uint16_t((1u << m) - 1);
+            uint8_t* e = block_table.data() + 16 * size_t(k);
+            e[0] = uint8_t(b); e[1] = uint8_t(n); e[2] = uint8_t(m);
+            put_u32(e + 4, m_before);
+            put_u64(e + 8, high.size());
+            m_before += uint32_t(m);
+        }
         std::vector<uint16_t> y(np, 0), hi3(np, 0);  // padding: y = 0
         for (uint32_t i = 0; i < real; ++i) {
             y[i] = ranked ? uint16_t(rank_of[x[first + i]]) : uint16_t(transform(x[first + i], b, n));
@@ -381,15 +417,22 @@ int encode(const void* in, int dtype, size_t count, bool have_params, int b, int
         }
     }
     table[g.nblocks] = a_total;
+    if (blockwise) {
+        uint8_t* e = block_table.data() + 16 * size_t(g.nblocks);
+        put_u32(e + 4, m_before);
+        put_u64(e + 8, high.size());
+    }
 
-    const Sections s = sections(dtype, count, g, n, m, a_total, ranked);
+    const Sections s = blockwise ? sections_blockwise(dtype, count, g, low.size(), high.size())
+                                 : sections(dtype, count, g, n, m, a_total, ranked);
     *out_size = s.total;
     if (capacity < s.total) return ERR_BUFFER_TOO_SMALL;
     std::memset(out, 0, s.total);
     std::memcpy(out, "ENEC", 4);
     put_u16(out + 4, 1);
     out[6] = uint8_t(dtype);
-    out[7] = ranked ? 1 : 0;  // variant: 0 = linear transform, 1 = frequency ranks
+    out[7] = blockwise ? 2 : ranked ? 1 : 0;  // variant: 0 = linear transform, 1 = frequency ranks, 2 = parameters per block
+    if (blockwise) { b = 0; n = 0; m = 0; }
     if (ranked) std::memcpy(out + s.unmap, unmap, 256);
     put_u64(out + 8, count);
     put_u32(out + 16, kBlock);
@@ -398,7 +441,8 @@ int encode(const void* in, int dtype, size_t count, bool have_params, int b, int
     put_u32(out + 28, g.total_groups);
     put_u32(out + 32, a_total);
     put_u64(out + 40, s.total);
-    for (size_t i = 0; i < table.size(); ++i) put_u32(out + s.table + 4 * i, table[i]);
+    if (blockwise) std::memcpy(out + s.table, block_table.data(), block_table.size());
+    else for (size_t i = 0; i < table.size(); ++i) put_u32(out + s.table + 4 * i, table[i]);
     if (!mask.empty()) std::memcpy(out + s.mask, mask.data(), mask.size());
     if (!low.empty()) std::memcpy(out + s.low, low.data(), low.size());
     if (!smhi.empty()) std::memcpy(out + s.smhi, smhi.data(), smhi.size());
@@ -423,31 +467,74 @@ int decode(const uint8_t* in, size_t in_size, int dtype, size_t count, void* out
     if (in[6] != dtype || get_u64(in + 8) != count || get_u32(in + 16) != kBlock || in[23] != kGroup)
         return ERR_BAD_STREAM;
     const int E = exp_bits(dtype);
-    const int b = in[20], n = in[21], m = in[22];
-    if (n < 1 || n > E || m < 1 || m > n || b >= (1 << E) || in[7] > 1) return ERR_BAD_STREAM;
-    const bool ranked = in[7] == 1;
+    int b = in[20], n = in[21], m = in[22];
+    if (in[7] > 2) return ERR_BAD_STREAM;
+    const bool ranked = in[7] == 1, blockwise = in[7] == 2;
+    if (!blockwise && (n < 1 || n > E || m < 1 || m > n || b >= (1 << E))) return ERR_BAD_STREAM;
+    if (blockwise && (b || n || m)) return ERR_BAD_STREAM;
     const Geometry g = geometry(count);
     const uint32_t a_total = get_u32(in + 32);
     if (get_u32(in + 24) != g.nblocks || get_u32(in + 28) != g.total_groups) return ERR_BAD_STREAM;
-    const Sections s = sections(dtype, count, g, n, m, a_total, ranked);
+    Sections s;
+    if (blockwise) {
+        // the block table's last entry holds the totals that fix the section sizes; the entries must chain
+        const size_t table_bytes = 16 * (size_t(g.nblocks) + 1);
+        if (in_size < kHeaderBytes + table_bytes) return ERR_BAD_STREAM;
+        const uint8_t* t = in + kHeaderBytes;
+        uint64_t m_sum = 0, high_sum = 0, low_sum = 0, wide_sum = 0;
+        for (uint32_t k = 0; k < g.nblocks; ++k) {
+            const uint8_t* e = t + 16 * size_t(k);
+            const int bb = e[0], nn = e[1], mm = e[2];
+            if (nn < 1 || nn > E || mm < 1 || mm > nn || bb >= (1 << E) || e[3]) return ERR_BAD_STREAM;
+            if (get_u32(e + 4) != m_sum || get_u64(e + 8) != high_sum) return ERR_BAD_STREAM;
+            const uint64_t next_high = get_u64(e + 24);
+            const uint64_t rec = uint64_t(2) * (nn - mm);
+            if (next_high < high_sum || (rec == 0 ? next_high != high_sum : (next_high - high_sum) % rec != 0)) return ERR_BAD_STREAM;
+            wide_sum += rec ? (next_high - high_sum) / rec : 0;
+            const uint32_t np = (k + 1 == g.nblocks) ? g.tail_padded : kBlock;
+            low_sum += uint64_t(np) * mm / 8;
+            m_sum += mm;
+            high_sum = next_high;
+        }
+        const uint8_t* last = t + 16 * size_t(g.nblocks);
+        if (last[0] || last[1] || last[2] || last[3] || get_u32(last + 4) != m_sum || get_u64(last + 8) != high_sum ||
+            wide_sum != a_total)
+            return ERR_BAD_STREAM;
+        s = sections_blockwise(dtype, count, g, low_sum, high_sum);
+    } else {
+        s = sections(dtype, count, g, n, m, a_total, ranked);
+    }
     if (get_u64(in + 40) != s.total || in_size < s.total) return ERR_BAD_STREAM;
-    if (get_u32(in + s.table + 4 * size_t(g.nblocks)) != a_total) return ERR_BAD_STREAM;
+    if (!blockwise && get_u32(in + s.table + 4 * size_t(g.nblocks)) != a_total) return ERR_BAD_STREAM;
 
-    const size_t rec_bytes = size_t(2) * (n - m);
+    size_t rec_bytes = blockwise ? 0 : size_t(2) * (n - m);
     for (uint32_t k = 0; k < g.nblocks; ++k) {
         size_t first = size_t(k) * kBlock;
         uint32_t real = (k + 1 == g.nblocks) ? g.tail_real : kBlock;
         uint32_t np = (k + 1 == g.nblocks) ? g.tail_padded : kBlock;
-        uint32_t rank = get_u32(in + s.table + 4 * size_t(k));  // records before this block
-        uint32_t next = get_u32(in + s.table + 4 * size_t(k + 1));
-        std::vector<uint16_t> y = alg2_unpack(in + s.low + size_t(k) * kBlock * m / 8, np, m);
+        size_t low_at = s.low + size_t(k) * kBlock * m / 8;
+        size_t high_at = s.high;     // of record number 0 (per tensor) or of the block's first record (per block)
+        uint32_t rank, next;         // records before this block and before the next one, in the units of high_at
+        if (blockwise) {
+            const uint8_t* e = in + s.table + 16 * size_t(k);
+            b = e[0]; n = e[1]; m = e[2];
+            rec_bytes = size_t(2) * (n - m);
+            low_at = s.low + size_t(2048) * get_u32(e + 4);
+            high_at = s.high + get_u64(e + 8);
+            rank = 0;
+            next = rec_bytes ? uint32_t((get_u64(e + 24) - get_u64(e + 8)) / rec_bytes) : 0;
+        } else {
+            rank = get_u32(in + s.table + 4 * size_t(k));
+            next = get_u32(in + s.table + 4 * size_t(k + 1));
+        }
+        std::vector<uint16_t> y = alg2_unpack(in + low_at, np, m);
         std::vector<uint16_t> hi3;
         if (dtype == 1) hi3 = alg2_unpack(in + s.smhi + size_t(k) * kBlock * 3 / 8, np, 3);
         for (uint32_t gi = 0; gi < np / kGroup; ++gi) {
             size_t gg = size_t(k) * (kBlock / kGroup) + gi;
             if ((in[s.mask + (gg >> 3)] >> (gg & 7)) & 1) {
                 if (rank >= next || n == m) return ERR_BAD_STREAM;
-                std::vector<uint16_t> hv = alg2_unpack(in + s.high + size_t(rank) * rec_bytes, kGroup, n - m);
+                std::vector<uint16_t> hv = alg2_unpack(in + high_at + size_t(rank) * rec_bytes, kGroup, n - m);
                 for (uint32_t j = 0; j < kGroup; ++j)
                     y[gi * kGroup + j] = uint16_t(y[gi * kGroup + j] | (hv[j] << m));
                 rank += 1;
@@ -526,6 +613,26 @@ size_t enec_oracle_max_compressed_size_ranked(int dtype, size_t count) {
 
 int enec_oracle_compress_ranked(const void* in, int dtype, size_t count, void* out, size_t capacity, size_t* out_size) {
     return encode(in, dtype, count, false, 0, 0, 0, static_cast<uint8_t*>(out), capacity, out_size, true);
+}
+
+// The block-wise variant: Sec. 5.5 on every block's own histogram; a 16-byte entry per block in place of the
+// prefix table. Worst case: the per-tensor worst case with the larger table (a block's low plane and records
+// together never exceed its elements times the exponent width, whatever its m).
+size_t enec_oracle_max_compressed_size_blockwise(int dtype, size_t count) {
+    if (!known_dtype(dtype) || (count >> 36)) return 0;
+    const int E = exp_bits(dtype);
+    const Geometry g = geometry(count);
+    size_t worst = 0;
+    for (int m = 1; m <= E; ++m) {
+        const Sections s = sections_blockwise(dtype, count, g, size_t(g.padded_count) * m / 8,
+                                              size_t(g.total_groups) * 2 * (E - m));
+        if (s.total > worst) worst = s.total;
+    }
+    return worst + 32;  // per-block m can leave both variable sections with up to 15 padding bytes each
+}
+
+int enec_oracle_compress_blockwise(const void* in, int dtype, size_t count, void* out, size_t capacity, size_t* out_size) {
+    return encode(in, dtype, count, false, 0, 0, 0, static_cast<uint8_t*>(out), capacity, out_size, false, true);
 }
 
 int enec_oracle_decompress(const void* in, size_t in_size, int dtype, size_t count, void* out) {

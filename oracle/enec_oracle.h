@@ -49,6 +49,11 @@ size_t enec_oracle_max_compressed_size(int dtype, size_t count);
 size_t enec_oracle_max_compressed_size_ranked(int dtype, size_t count);
 int enec_oracle_compress_ranked(const void* in, int dtype, size_t count, void* out, size_t capacity, size_t* out_size);
 
+/* The block-wise variant (Sec. 5.5 run on every block's own histogram): header byte 7 = 2; a block table of
+ * 16-byte entries {b, n, m, 0, u32 sum of m before, u64 record bytes before} replaces the prefix table. */
+size_t enec_oracle_max_compressed_size_blockwise(int dtype, size_t count);
+int enec_oracle_compress_blockwise(const void* in, int dtype, size_t count, void* out, size_t capacity, size_t* out_size);
+
 int enec_oracle_compress(const void* in, int dtype, size_t count, void* out, size_t capacity,
                          size_t* out_size);
 int enec_oracle_compress_with_params(const void* in, int dtype, size_t count, int b, int n, int m,

@@ -50,6 +50,10 @@ def lib():
         L.enec_oracle_compress.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_void_p, C.c_size_t,
                                            C.POINTER(C.c_size_t)]
         L.enec_oracle_compress.restype = C.c_int
+        L.enec_oracle_max_compressed_size_blockwise.argtypes = [C.c_int, C.c_size_t]
+        L.enec_oracle_max_compressed_size_blockwise.restype = C.c_size_t
+        L.enec_oracle_compress_blockwise.argtypes = L.enec_oracle_compress.argtypes
+        L.enec_oracle_compress_blockwise.restype = C.c_int
         L.enec_oracle_compress_with_params.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_int,
                                                        C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
         L.enec_oracle_compress_with_params.restype = C.c_int
@@ -142,6 +146,22 @@ def compress_ranked(words, dtype):
     out = np.empty(cap, dtype=np.uint8)
     size = C.c_size_t(0)
     st = lib().enec_oracle_compress_ranked(words.ctypes.data, dtype, words.size, out.ctypes.data, cap, C.byref(size))
+    if st != 0:
+        raise OracleError(st)
+    return out[:size.value].copy()
+
+
+def max_compressed_size_blockwise(dtype, count):
+    return lib().enec_oracle_max_compressed_size_blockwise(dtype, count)
+
+
+def compress_blockwise(words, dtype):
+    """The block-wise variant of compress(): every block chooses its own (b, n, m)."""
+    words = np.ascontiguousarray(words, dtype=np.uint32 if dtype == FP32 else np.uint16).reshape(-1)
+    cap = max_compressed_size_blockwise(dtype, words.size)
+    out = np.empty(cap, dtype=np.uint8)
+    size = C.c_size_t(0)
+    st = lib().enec_oracle_compress_blockwise(words.ctypes.data, dtype, words.size, out.ctypes.data, cap, C.byref(size))
     if st != 0:
         raise OracleError(st)
     return out[:size.value].copy()

@@ -60,6 +60,8 @@ def lib():
         L.enec_compress_batched.restype = C.c_int
         L.enec_launch_count.argtypes = []
         L.enec_launch_count.restype = C.c_uint64
+        L.enec_allocation_count.argtypes = []
+        L.enec_allocation_count.restype = C.c_uint64
         L.enec_version.argtypes = []
         L.enec_version.restype = C.c_int
         _LIB = L
@@ -141,6 +143,10 @@ def enec_compress_batched(items, dt, d_out_sizes=None, d_status=None) -> int:
 
 def enec_launch_count() -> int:
     return lib().enec_launch_count()
+
+
+def enec_allocation_count() -> int:
+    return lib().enec_allocation_count()
 
 
 # ---- convenience wrappers (allocation with torch, status check) --------------------------------------

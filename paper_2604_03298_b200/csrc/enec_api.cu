@@ -21,14 +21,18 @@ struct DeviceInfo {
     bool batch_attr_set[3] = {false, false, false};
 };
 
-static DeviceInfo& device_info(int dev) {
+// Per-device facts, for device ordinals below kMaxDevices (null beyond: the caller fails with ENEC_ERR_CUDA).
+static DeviceInfo* device_info(int dev) {
     static std::mutex mu;
-    static DeviceInfo infos[64];
+    static DeviceInfo infos[kMaxDevices];
+    if (dev < 0 || dev >= kMaxDevices) return nullptr;
     std::lock_guard<std::mutex> lock(mu);
-    DeviceInfo& d = infos[dev & 63];
+    DeviceInfo& d = infos[dev];
     if (d.sms == 0) cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev);
-    return d;
+    return &d;
 }
+
+std::atomic<uint64_t> g_allocations{0};  // cudaMalloc calls the library has made (enec_allocation_count)
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -56,6 +60,7 @@ static enec_status grow(ScratchArea& a, size_t need) {
     while (bytes < need) bytes *= 2;
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) return ENEC_ERR_CUDA;
+    g_allocations.fetch_add(1, std::memory_order_relaxed);
     a.ptr = static_cast<uint8_t*>(p);
     a.bytes = bytes;
     a.needs_clear = true;
@@ -194,7 +199,9 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
     }
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
-    DeviceInfo& info = device_info(dev);
+    DeviceInfo* found = device_info(dev);
+    if (!found) return ENEC_ERR_CUDA;
+    DeviceInfo& info = *found;
     const Geometry g = make_geometry(count);
     const size_t need = kControlBytes + size_t(g.nblocks) * sizeof(unsigned long long);
     // the scratch area carries state from call to call, which a replayed recording would not see
@@ -235,8 +242,8 @@ static_assert(kNoAllocScratchBytes == ENEC_NOALLOC_SCRATCH_BYTES, "the header st
 // Device address of the scratch on the current device, looked up once per device.
 static enec_status noalloc_scratch(int dev, uint8_t** out) {
     static std::mutex mu;
-    static uint8_t* addr[64] = {};
-    if (dev < 0 || dev >= 64) return ENEC_ERR_CUDA;
+    static uint8_t* addr[kMaxDevices] = {};
+    if (dev < 0 || dev >= kMaxDevices) return ENEC_ERR_CUDA;
     std::lock_guard<std::mutex> lock(mu);
     if (!addr[dev]) {
         void* p = nullptr;
@@ -318,7 +325,25 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
         if (total >> 31) return ENEC_ERR_INVALID_ARG;  // block indices are 32-bit
     }
     prefix[n_items] = uint32_t(total);
-    if (total == 0) return ENEC_OK;
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return ENEC_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone && uint32_t(n_items) > kInlineJobs) {
+        // A recording must hold neither a copy from this call's host memory nor the library's scratch: lists of
+        // up to kInlineJobs tensors travel inside the launch parameters, so a longer list becomes several launches.
+        for (int first = 0; first < n_items; first += int(kInlineJobs)) {
+            const int n = n_items - first < int(kInlineJobs) ? n_items - first : int(kInlineJobs);
+            DecodeBatch part;
+            part.jobs = nullptr;
+            part.prefix = nullptr;
+            part.n_jobs = uint32_t(n);
+            part.total_blocks = prefix[first + n] - prefix[first];
+            for (int i = 0; i < n; ++i) part.inline_jobs[i] = jobs[first + i];
+            for (int i = 0; i <= n; ++i) part.inline_prefix[i] = prefix[first + i] - prefix[first];
+            const enec_status st = launch_decode_any(dt, part, d_status, stream, false);
+            if (st != ENEC_OK) return st;
+        }
+        return ENEC_OK;
+    }
     DecodeBatch batch;
     batch.n_jobs = uint32_t(n_items);
     batch.total_blocks = uint32_t(total);
@@ -379,7 +404,13 @@ enec_status enec_compress_batched(const enec_batch_item* h_items, int n_items, e
     }
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
-    DeviceInfo& info = device_info(dev);
+    DeviceInfo* found = device_info(dev);
+    if (!found) return ENEC_ERR_CUDA;
+    DeviceInfo& info = *found;
+    // the call clears and fills scratch from host memory that does not outlive it: not something to record
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return ENEC_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) return ENEC_ERR_INVALID_ARG;
     unsigned long long* sizes = reinterpret_cast<unsigned long long*>(d_out_sizes);
     // device scratch of the call: [ticket | control words per tensor | state word per block | jobs | prefix | units];
     // everything in front of the tables is cleared, the tables are copied from the host
@@ -470,7 +501,9 @@ enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count,
     uint8_t* scratch = nullptr;
     const enec_status st = noalloc_scratch(dev, &scratch);
     if (st != ENEC_OK) return st;
-    DeviceInfo& info = device_info(dev);
+    DeviceInfo* found = device_info(dev);
+    if (!found) return ENEC_ERR_CUDA;
+    DeviceInfo& info = *found;
     const Geometry g = make_geometry(count);
     // the area keeps the previous call's words: histogram, ticket, flags and state words start at zero
     const size_t used = kControlBytes + size_t(g.nblocks) * sizeof(unsigned long long);
@@ -491,6 +524,8 @@ enec_status enec_compress_noalloc(const void* d_in, enec_dtype dt, size_t count,
 }
 
 uint64_t enec_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+uint64_t enec_allocation_count(void) { return g_allocations.load(std::memory_order_relaxed); }
 
 int enec_version(void) { return 100; }
 

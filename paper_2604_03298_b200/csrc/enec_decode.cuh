@@ -696,14 +696,18 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     }
     __syncthreads();
     pdl_wait();  // nothing above uses what it read from global memory, except as prefetch addresses
-    if (batch.total_blocks == 0) {  // nothing to decode: only check the header of a single empty tensor
-        if (threadIdx.x == 0 && blockIdx.x == 0 && batch.jobs == nullptr && batch.n_jobs == 1) {
-            JobCtx jc;
-            const int err = load_job<DT, MAPPED>(batch.inline_jobs[0], jc);
-            if (err) report(status, err);
+    if (blockIdx.x == 0) {
+        // tensors without elements have no block that would bring their header before the loader: check them here
+        const DecodeJob* all_jobs = batch.jobs ? batch.jobs : batch.inline_jobs;
+        for (uint32_t q = threadIdx.x; q < batch.n_jobs; q += blockDim.x) {
+            if (all_jobs[q].count == 0) {
+                JobCtx jc;
+                const int err = load_job<DT, MAPPED>(all_jobs[q], jc);
+                if (err) report(status, err);
+            }
         }
-        return;
     }
+    if (batch.total_blocks == 0) return;
 
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lane = threadIdx.x & 31;

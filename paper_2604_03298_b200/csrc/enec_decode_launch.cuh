@@ -13,20 +13,23 @@ struct DecodeDevice {
     int sms = 0;
     bool attr_set[3] = {false, false, false};
 };
-inline DecodeDevice& decode_device(int dev) {
+inline DecodeDevice* decode_device(int dev) {
     static std::mutex mu;
-    static DecodeDevice infos[64];
+    static DecodeDevice infos[kMaxDevices];
+    if (dev < 0 || dev >= kMaxDevices) return nullptr;
     std::lock_guard<std::mutex> lock(mu);
-    DecodeDevice& d = infos[dev & 63];
+    DecodeDevice& d = infos[dev];
     if (d.sms == 0) cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev);
-    return d;
+    return &d;
 }
 
 template <int DT>
 inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked = false) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
-    DecodeDevice& info = decode_device(dev);
+    DecodeDevice* found = decode_device(dev);
+    if (!found) return ENEC_ERR_CUDA;
+    DecodeDevice& info = *found;
     if (!info.attr_set[DT]) {
         if (cudaFuncSetAttribute(enec_decode_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(kDecodeSmemBytes)) != cudaSuccess ||

@@ -10,6 +10,7 @@
 namespace enec {
 
 extern std::atomic<uint64_t> g_launches;  // kernels launched by the library (enec_launch_count)
+constexpr int kMaxDevices = 64;  // device ordinals the per-device tables cover; calls on others fail with ENEC_ERR_CUDA
 
 struct DecodeBatch;
 // Launches the decode kernel instance for dt (and for the frequency-rank variant when ranked) over `batch`.

@@ -24,7 +24,7 @@ def declared_functions():
 def test_header_declares_the_expected_entry_points():
     names = declared_functions()
     for want in ("enec_max_compressed_size", "enec_compress", "enec_compress_with_params", "enec_decompress",
-                 "enec_compress_batched", "enec_decompress_batched", "enec_compress_noalloc", "enec_launch_count",
+                 "enec_compress_batched", "enec_decompress_batched", "enec_compress_noalloc", "enec_launch_count", "enec_allocation_count",
                  "enec_version"):
         assert want in names
 

@@ -190,3 +190,58 @@ def test_compress_batched_argument_checks():
     assert enec.enec_compress_batched([(src, dst, 4096, cap - 1)], 0) == -3
     assert enec.enec_compress_batched([(src[1:], dst, 4000, cap)], 0) == -1
     torch.cuda.synchronize()
+
+
+def test_batched_decompress_checks_members_without_elements():
+    """A member with count 0 has an 80-byte stream and no block: its header must still be looked at, alone or among
+    tensors that do have blocks, as enec_decompress does for an empty tensor."""
+    import paper_2604_03298_b200 as enec
+    empty = torch.empty(0, dtype=torch.bfloat16, device="cuda")
+    full = (torch.randn(40000, device="cuda") * 0.02).to(torch.bfloat16)
+    s_empty, s_full = enec.compress_tensor(empty), enec.compress_tensor(full)
+    assert s_empty.numel() == 80
+    out = torch.empty_like(full)
+    none = torch.empty(16, dtype=torch.bfloat16, device="cuda")
+    for streams in ([s_empty.clone()], [s_full, s_empty.clone()]):
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        items = [(s, s.numel(), out if s.numel() > 80 else none, full.numel() if s.numel() > 80 else 0) for s in streams]
+        assert enec.enec_decompress_batched(items, 0, status) == 0
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        streams[-1][0] = 0x58           # damage the empty member's magic
+        assert enec.enec_decompress_batched(items, 0, status) == 0
+        torch.cuda.synchronize()
+        assert int(status.item()) == -4
+    assert torch.equal(out.view(torch.int16), full.view(torch.int16))
+
+
+def test_batched_calls_under_stream_capture():
+    """A batch of more than 16 tensors recorded into a CUDA graph: the decompress call records launches whose
+    tensor lists travel in their parameters (nothing of the call's host memory or the library's scratch is in the
+    graph), and replays bit for bit after the outputs were wiped; the compress call is refused."""
+    import paper_2604_03298_b200 as enec
+    g = torch.Generator(device="cuda").manual_seed(77)
+    raw = [(torch.randn(16384 * 2 + 100 * i + 5, generator=g, device="cuda") * 0.02).to(torch.bfloat16) for i in range(17)]
+    streams = [enec.compress_tensor(t) for t in raw]
+    outs = [torch.zeros_like(t) for t in raw]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    items = enec.make_batch([(s, o, t.numel(), s.numel()) for s, o, t in zip(streams, outs, raw)])
+    comp_items = enec.make_batch([(t, torch.empty(enec.enec_max_compressed_size(0, t.numel()), dtype=torch.uint8, device="cuda"),
+                                   t.numel(), enec.enec_max_compressed_size(0, t.numel())) for t in raw])
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    before = enec.enec_launch_count()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            assert enec.enec_compress_batched(comp_items, 0, None, status) == -1
+            assert enec.enec_decompress_batched(items, 0, status) == 0
+    assert enec.enec_launch_count() - before == 2      # 16 + 1 tensors
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for o, t in zip(outs, raw):
+            assert torch.equal(o.view(torch.int16), t.view(torch.int16))

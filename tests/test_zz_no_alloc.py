@@ -65,3 +65,25 @@ def test_noalloc_refuses_what_does_not_fit_its_array():
     assert enec.enec_compress_noalloc(small, enec.BF16, 64, dst, 10) == -3
     assert enec.enec_compress_noalloc(small, 5, 64, dst, 4096) == -2
     torch.cuda.synchronize()
+
+
+def test_noalloc_makes_no_allocation_where_enec_compress_does():
+    """What the entry point is for: on a stream the library has never seen, enec_compress takes scratch from
+    cudaMalloc (the library counts its calls) and enec_compress_noalloc does not."""
+    import paper_2604_03298_b200 as enec
+    from paper_2604_03298_b200 import synth
+    t = synth.make_tensor(synth.TensorSpec("d", torch.bfloat16, (16384 * 5 + 11,), "normal", 0.0, 0.02, 94), "cuda")
+    torch.cuda.synchronize()
+    fresh = torch.cuda.Stream()
+    with torch.cuda.stream(fresh):
+        before = enec.enec_allocation_count()
+        a = _compress(enec.enec_compress_noalloc, t)
+        b = _compress(enec.enec_compress_noalloc, t)
+        assert enec.enec_allocation_count() == before
+        c = _compress(enec.enec_compress, t)
+        assert enec.enec_allocation_count() == before + 1
+    torch.cuda.synchronize()
+    n = int(c[1].item())
+    for buf, size, status, cap in (a, b):
+        assert int(status.item()) == 0 and int(size.item()) == n
+        assert torch.equal(buf[:n], c[0][:n])
