@@ -625,3 +625,121 @@ def test_ranked_is_a_little_smaller_on_gaussian_weights(oracle):
     w = (torch.randn(1 << 20, generator=torch.Generator().manual_seed(5)) * 0.02).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     linear, ranked = oracle.compress(w, 0).size, oracle.compress_ranked(w, 0).size
     assert ranked < linear < ranked * 1.03
+
+
+# ---------------------------------------------------------------- block-wise variant (Sec. 5.5 per block)
+def _blockwise_table(s, nblocks):
+    """(b, n, m, sum of m before, record bytes before) of every entry of a block-wise stream's block table."""
+    t = s[64:64 + 16 * (nblocks + 1)]
+    return [(int(t[16 * k]), int(t[16 * k + 1]), int(t[16 * k + 2]), int(t[16 * k + 4:16 * k + 8].view(np.uint32)[0]),
+             int(t[16 * k + 8:16 * k + 16].view(np.uint64)[0])) for k in range(nblocks + 1)]
+
+
+def test_blockwise_stream_hand(oracle):
+    fx = read_fixture("stream_hand_blockwise.txt")
+    base = int(fx["block0_word_base"][0], 16)
+    words = np.concatenate([(base + (np.arange(16384) & 127)).astype(np.uint16),
+                            np.array([int(t, 16) for t in fx["block1_words"][0].split()], dtype=np.uint16)])
+    assert words.size == int(fx["count"][0])
+    expect = np.concatenate([hexbytes(fx["header"][0]), hexbytes(fx["table"][0]),
+                             np.zeros(int(fx["mask_zero_bytes"][0]), np.uint8),
+                             np.zeros(int(fx["low_zero_bytes"][0]), np.uint8), hexbytes(fx["low_tail"][0]),
+                             (np.arange(16384) % 128).astype(np.uint8), hexbytes(fx["sm_block1"][0])])
+    got = oracle.compress_blockwise(words, 0)
+    assert got.size == 18720 and got.tolist() == expect.tolist()
+    assert oracle.decompress(got, 0, words.size).tolist() == words.tolist()
+
+
+def test_blockwise_equals_the_per_tensor_stream_when_all_blocks_agree(oracle):
+    # every block holds the same multiset of exponents, so every block's search gives the tensor's (b, n, m):
+    # mask, low plane, sign/mantissa bytes and records must then be the per-tensor stream's, byte for byte
+    rng = np.random.default_rng(51)
+    nblocks = 3
+    one = np.clip(np.round(rng.normal(121, 2.0, 16384)), 100, 130).astype(np.uint16)
+    x = np.concatenate([rng.permutation(one) for _ in range(nblocks)])
+    words = ((x << 7) | rng.integers(0, 128, x.size).astype(np.uint16)).astype(np.uint16)
+    a = oracle.compress(words, 0)
+    b = oracle.compress_blockwise(words, 0)
+    params = (int(a[20]), int(a[21]), int(a[22]))
+    table = _blockwise_table(b, nblocks)
+    assert [e[:3] for e in table[:nblocks]] == [params] * nblocks
+    assert [e[3] for e in table] == [k * params[2] for k in range(nblocks + 1)]
+    per_tensor_table = a[64:64 + 4 * (nblocks + 1)].view(np.uint32)
+    assert [e[4] for e in table] == [int(v) * 2 * (params[1] - params[2]) for v in per_tensor_table]
+    a16 = lambda v: (v + 15) // 16 * 16
+    assert a[64 + a16(4 * (nblocks + 1)):].tolist() == b[64 + a16(16 * (nblocks + 1)):].tolist()
+    assert b[7] == 2 and not b[20:23].any() and b[32:36].tolist() == a[32:36].tolist()
+    assert int(b[40:48].view(np.uint64)[0]) == b.size == a.size + a16(16 * (nblocks + 1)) - a16(4 * (nblocks + 1))
+
+
+def test_blockwise_parameters_are_each_blocks_own_search(oracle):
+    # blocks drawn at different scales choose different parameters; each must be what the search of Sec. 5.5 gives
+    # on that block's histogram alone, the offsets must chain, and the size must follow the closed form
+    import torch
+    g = torch.Generator().manual_seed(52)
+    parts = [torch.randn(16384, generator=g) * 0.02, torch.randn(16384, generator=g) * 3.0, torch.zeros(16384),
+             torch.randn(5000, generator=g) * 1e-3]
+    parts[2][::7] = 1.0                      # exact zeros next to ones: exponents 0 and 127, n = 8
+    words = torch.cat(parts).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    s = oracle.compress_blockwise(words, 0)
+    nblocks = 4
+    table = _blockwise_table(s, nblocks)
+    m_sum = high = wide_total = 0
+    low_bytes = 0
+    for k in range(nblocks):
+        blk = words[k * 16384:(k + 1) * 16384]
+        hist = np.bincount((blk >> 7) & 0xFF, minlength=256).astype(np.uint64)
+        b, n, m, _, _ = oracle.param_search(hist, 8)
+        assert table[k][:3] == (b, n, m), k
+        assert table[k][3] == m_sum and table[k][4] == high
+        y = (b - ((blk.astype(np.int64) >> 7) & 0xFF)) % (1 << n)
+        padded = 16384 if k < 3 else 8192
+        y = np.concatenate([y, np.zeros(padded - y.size, np.int64)]).reshape(-1, 16)
+        wide = int((np.bitwise_or.reduce(y, axis=1) >> m != 0).sum())
+        wide_total += wide
+        high += wide * 2 * (n - m)
+        low_bytes += padded * m // 8
+        m_sum += m
+    assert table[nblocks] == (0, 0, 0, m_sum, high)
+    assert len({e[:3] for e in table[:nblocks]}) >= 3
+    assert int(s[32:36].view(np.uint32)[0]) == wide_total
+    a16 = lambda v: (v + 15) // 16 * 16
+    groups = (3 * 16384 + 8192) // 16
+    assert s.size == 64 + a16(16 * 5) + a16((groups + 7) // 8) + a16(low_bytes) + a16(words.size) + a16(high)
+    assert s.size <= oracle.max_compressed_size_blockwise(0, words.size)
+    assert np.array_equal(oracle.decompress(s, 0, words.size), words)
+    # where one stray zero forces n = 8 on the whole tensor, the blocks without it keep their narrow codes
+    assert s.size < oracle.compress(words, 0).size
+
+
+@pytest.mark.parametrize("dt", [0, 1, 2])
+def test_blockwise_roundtrip_patterns_and_tails(oracle, dt):
+    rng = np.random.default_rng(53 + dt)
+    if dt == 2:
+        full = rng.integers(0, 1 << 32, 70000, dtype=np.uint64).astype(np.uint32)
+    else:
+        full = rng.permutation(1 << 16).astype(np.uint16)
+    s = oracle.compress_blockwise(full, dt)
+    assert s.size <= oracle.max_compressed_size_blockwise(dt, full.size)
+    assert np.array_equal(oracle.decompress(s, dt, full.size), full)
+    for count in (0, 1, 15, 16, 17, 1000, 16384, 16385, 2 * 16384 + 4097):
+        w = full[:count]
+        s = oracle.compress_blockwise(w, dt)
+        assert s.size % 16 == 0 and s.size <= oracle.max_compressed_size_blockwise(dt, count)
+        assert np.array_equal(oracle.decompress(s, dt, count), w)
+    worst = np.tile(np.array([0x0000, 0x7F80] * 8, np.uint16), 2048 * 2 + 3) if dt == 0 else None
+    if worst is not None:    # every group wide with n = 8 in every block: the size bound must hold
+        s = oracle.compress_blockwise(worst, 0)
+        assert s.size <= oracle.max_compressed_size_blockwise(0, worst.size)
+
+
+def test_blockwise_decoder_rejects_damaged_tables(oracle):
+    rng = np.random.default_rng(54)
+    words = rng.integers(0x3A00, 0x3FFF, 40000).astype(np.uint16)
+    s = oracle.compress_blockwise(words, 0)
+    assert np.array_equal(oracle.decompress(s, 0, words.size), words)
+    for off, val in ((7, 3), (20, 1), (64 + 1, 9), (64 + 2, 0), (64 + 16 + 4, 7), (64 + 16 + 8, 1), (64 + 48 + 4, 0)):
+        bad = s.copy()
+        bad[off] = val
+        with pytest.raises(oracle.OracleError):
+            oracle.decompress(bad, 0, words.size)
