@@ -112,6 +112,28 @@ enec_status enec_compress_ranked(const void* d_in, enec_dtype dt, size_t count, 
 enec_status enec_decompress_ranked(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
                                    int* d_status, enec_stream_t stream);
 
+/*
+ * The block-wise variant of enec_compress, kept for the ablation: the search of Sec. 5.5 (Eq. 1-5) runs on the
+ * exponent histogram of every 16384-element block instead of the tensor's, so each block is coded with its own
+ * (b, n, m). (Sec. 6.4 and Table 6 measure how little is lost by sharing parameters; this variant measures the
+ * other end of that trade on the GPU.) The stream has header byte 7 = 2 and header bytes 20..22 zero; in place of
+ * the prefix table it carries a block table of 16-byte entries, one per block plus one with the totals:
+ *   byte 0 b, byte 1 n, byte 2 m, byte 3 zero,
+ *   bytes 4..7   u32: sum of m over the blocks before (the block's low plane starts 2048 x that many bytes into
+ *                the low-plane section),
+ *   bytes 8..15  u64: bytes of wide-group records before the block's first record;
+ * header bytes 32..35 hold the number of wide groups of the tensor. Every other section is laid out as by
+ * enec_compress. out_capacity must be at least enec_max_compressed_size_blockwise(dt, count). The arguments,
+ * the scratch rule, the stream-capture rule (refused with ENEC_ERR_INVALID_ARG) and the error behaviour are those
+ * of enec_compress. Such a stream is decoded by enec_decompress_blockwise (same arguments as enec_decompress);
+ * every decompress call reports ENEC_ERR_BAD_STREAM in *d_status for a stream of another variant.
+ */
+size_t enec_max_compressed_size_blockwise(enec_dtype dt, size_t count);
+enec_status enec_compress_blockwise(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                                    size_t* d_out_size, int* d_status, enec_stream_t stream);
+enec_status enec_decompress_blockwise(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
+                                      int* d_status, enec_stream_t stream);
+
 /* One tensor of a batch. All pointers are device pointers. */
 typedef struct {
     const void* d_in;    /* decompress: stream; compress: raw values            */

@@ -46,6 +46,10 @@ def lib():
         L.enec_compress_ranked.restype = C.c_int
         L.enec_max_compressed_size_ranked.argtypes = [C.c_int, C.c_size_t]
         L.enec_max_compressed_size_ranked.restype = C.c_size_t
+        L.enec_compress_blockwise.argtypes = L.enec_compress.argtypes
+        L.enec_compress_blockwise.restype = C.c_int
+        L.enec_max_compressed_size_blockwise.argtypes = [C.c_int, C.c_size_t]
+        L.enec_max_compressed_size_blockwise.restype = C.c_size_t
         L.enec_compress_with_params.argtypes = [C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_int,
                                                 C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
         L.enec_compress_with_params.restype = C.c_int
@@ -54,6 +58,8 @@ def lib():
         L.enec_decompress.restype = C.c_int
         L.enec_decompress_ranked.argtypes = L.enec_decompress.argtypes
         L.enec_decompress_ranked.restype = C.c_int
+        L.enec_decompress_blockwise.argtypes = L.enec_decompress.argtypes
+        L.enec_decompress_blockwise.restype = C.c_int
         L.enec_decompress_batched.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.enec_decompress_batched.restype = C.c_int
         L.enec_compress_batched.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -102,6 +108,21 @@ def enec_compress_ranked(d_in, dt, count, d_out, out_capacity, d_out_size=None, 
     """The frequency-rank variant of enec_compress (ablation): same arguments, 256 bytes more capacity."""
     return lib().enec_compress_ranked(_ptr(d_in), dt, count, _ptr(d_out), out_capacity, _ptr(d_out_size),
                                       _ptr(d_status), _stream())
+
+
+def enec_max_compressed_size_blockwise(dt: int, count: int) -> int:
+    return lib().enec_max_compressed_size_blockwise(dt, count)
+
+
+def enec_compress_blockwise(d_in, dt, count, d_out, out_capacity, d_out_size=None, d_status=None) -> int:
+    """The block-wise variant of enec_compress (ablation): every 16384-element block gets its own (b, n, m)."""
+    return lib().enec_compress_blockwise(_ptr(d_in), dt, count, _ptr(d_out), out_capacity, _ptr(d_out_size),
+                                         _ptr(d_status), _stream())
+
+
+def enec_decompress_blockwise(d_in, in_size, dt, count, d_out, d_status=None) -> int:
+    """Decompresses a stream written by enec_compress_blockwise."""
+    return lib().enec_decompress_blockwise(_ptr(d_in), in_size, dt, count, _ptr(d_out), _ptr(d_status), _stream())
 
 
 def enec_compress_with_params(d_in, dt, count, b, n, m, d_out, out_capacity, d_out_size=None, d_status=None) -> int:

@@ -8,6 +8,7 @@
 
 #include "enec_decode.cuh"
 #include "enec_encode.cuh"
+#include "enec_blockwise.cuh"
 #include "enec_launch.cuh"
 
 namespace enec {
@@ -19,6 +20,7 @@ struct DeviceInfo {
     bool hist_attr_set[3] = {false, false, false};
     bool encode_attr_set[3] = {false, false, false};
     bool batch_attr_set[3] = {false, false, false};
+    bool blockwise_attr_set[3] = {false, false, false};
 };
 
 // Per-device facts, for device ordinals below kMaxDevices (null beyond: the caller fails with ENEC_ERR_CUDA).
@@ -46,7 +48,7 @@ struct ScratchArea {
     bool needs_clear = true;  // compressor areas: fresh memory, a wrapped epoch or a launch that failed
 };
 
-enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1, kScratchCompressBatch = 2 };
+enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1, kScratchCompressBatch = 2, kScratchBlockwise = 3 };
 
 static std::mutex g_scratch_mu;
 static ScratchArea& scratch_area(int dev, cudaStream_t stream, ScratchKind kind) {
@@ -254,6 +256,102 @@ static enec_status noalloc_scratch(int dev, uint8_t** out) {
     return ENEC_OK;
 }
 
+// ---- the block-wise variant ------------------------------------------------------------------------
+
+// The counter of finished blocks: zeroed when the area is new or after a call on it failed to launch; the
+// kernel that uses it leaves it at zero.
+static enec_status lease_blockwise_counter(int dev, cudaStream_t stream, uint32_t** out) {
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    ScratchArea& a = scratch_area(dev, stream, kScratchBlockwise);
+    const enec_status st = grow(a, 256);
+    if (st != ENEC_OK) return st;
+    if (a.needs_clear) {
+        if (cudaMemsetAsync(a.ptr, 0, 256, stream) != cudaSuccess) return ENEC_ERR_CUDA;
+        a.needs_clear = false;
+    }
+    *out = reinterpret_cast<uint32_t*>(a.ptr);
+    return ENEC_OK;
+}
+
+template <int DT>
+static enec_status launch_blockwise(const BlockwiseJob& job, uint32_t nblocks, int* d_status, DeviceInfo& info,
+                                    cudaStream_t stream) {
+    if (!info.blockwise_attr_set[DT]) {
+        if (cudaFuncSetAttribute(enec_block_params_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(HistShape<DT>::kBytes)) != cudaSuccess ||
+            cudaFuncSetAttribute(enec_pack_blocks_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(kPackSmemBytes)) != cudaSuccess)
+            return ENEC_ERR_CUDA;
+        info.blockwise_attr_set[DT] = true;
+    }
+    uint32_t grid = uint32_t(info.sms) * 3;
+    if (grid > nblocks) grid = nblocks;
+    cudaError_t err = launch_pdl(enec_block_params_kernel<DT>, grid, kBlockwiseThreads, HistShape<DT>::kBytes, stream, job,
+                                 d_status);
+    if (err != cudaSuccess) return ENEC_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    grid = uint32_t(info.sms) * 4;
+    if (grid > nblocks) grid = nblocks;
+    err = launch_pdl(enec_pack_blocks_kernel<DT>, grid, kBlockwiseThreads, kPackSmemBytes, stream, job, d_status);
+    if (err != cudaSuccess) return ENEC_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ENEC_OK;
+}
+
+static size_t max_size_blockwise(enec_dtype dt, size_t count) {
+    if (!known_dtype(dt) || (uint64_t(count) >> 36)) return 0;
+    const int E = exp_bits(dt);
+    const Geometry g = make_geometry(count);
+    // a block's low plane and records together are largest when all its groups are wide with n = E; the two
+    // variable sections each end in up to 15 bytes of padding
+    uint64_t worst = 0;
+    for (int m = 1; m <= E; ++m) {
+        const uint64_t t = make_sections_blockwise(dt, count, g, g.padded_count * uint64_t(m) / 8,
+                                                   uint64_t(g.total_groups) * 2 * uint64_t(E - m)).total;
+        if (t > worst) worst = t;
+    }
+    return size_t(worst + 32);
+}
+
+static enec_status compress_blockwise(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                                      size_t* d_out_size, int* d_status, cudaStream_t stream) {
+    if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
+    if ((!d_in && count) || !d_out || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out) ||
+        (reinterpret_cast<uintptr_t>(d_out_size) & 7))
+        return ENEC_ERR_INVALID_ARG;
+    if (out_capacity < max_size_blockwise(dt, count)) return ENEC_ERR_BUFFER_TOO_SMALL;
+    unsigned long long* out_size = reinterpret_cast<unsigned long long*>(d_out_size);
+    if (count == 0) {
+        enec_encode_empty_kernel<<<1, 32, 0, stream>>>(static_cast<uint8_t*>(d_out), int(dt), 0, 0, 0, out_size, 2);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
+    DeviceInfo* found = device_info(dev);
+    if (!found) return ENEC_ERR_CUDA;
+    // the counter carries state from call to call, which a replayed recording would not see
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return ENEC_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) return ENEC_ERR_INVALID_ARG;
+    BlockwiseJob job;
+    job.in = static_cast<const uint16_t*>(d_in);
+    job.out = static_cast<uint8_t*>(d_out);
+    job.count = count;
+    job.out_size = out_size;
+    enec_status st = lease_blockwise_counter(dev, stream, &job.done);
+    if (st != ENEC_OK) return st;
+    const uint32_t nblocks = make_geometry(count).nblocks;
+    st = dt == ENEC_BF16   ? launch_blockwise<ENEC_BF16>(job, nblocks, d_status, *found, stream)
+         : dt == ENEC_FP16 ? launch_blockwise<ENEC_FP16>(job, nblocks, d_status, *found, stream)
+                           : launch_blockwise<ENEC_FP32>(job, nblocks, d_status, *found, stream);
+    if (st != ENEC_OK) {
+        std::lock_guard<std::mutex> lock(g_scratch_mu);
+        scratch_area(dev, stream, kScratchBlockwise).needs_clear = true;
+    }
+    return st;
+}
+
 }  // namespace enec
 
 using namespace enec;
@@ -273,7 +371,7 @@ size_t enec_max_compressed_size(enec_dtype dt, size_t count) {
 }
 
 static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
-                                  int* d_status, cudaStream_t stream, bool ranked) {
+                                  int* d_status, cudaStream_t stream, bool ranked, bool blockwise = false) {
     if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if (!d_in || (!d_out && count) || (uint64_t(count) >> 36) || !aligned16(d_in) || !aligned16(d_out))
         return ENEC_ERR_INVALID_ARG;
@@ -282,6 +380,7 @@ static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype d
     batch.jobs = nullptr;
     batch.prefix = nullptr;
     batch.n_jobs = 1;
+    batch.blockwise = blockwise ? 1 : 0;
     batch.total_blocks = make_geometry(count).nblocks;
     batch.inline_jobs[0] = DecodeJob{static_cast<const uint8_t*>(d_in), static_cast<uint16_t*>(d_out), uint64_t(count),
                                      uint64_t(in_size)};
@@ -336,6 +435,7 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
             part.jobs = nullptr;
             part.prefix = nullptr;
             part.n_jobs = uint32_t(n);
+            part.blockwise = 0;
             part.total_blocks = prefix[first + n] - prefix[first];
             for (int i = 0; i < n; ++i) part.inline_jobs[i] = jobs[first + i];
             for (int i = 0; i <= n; ++i) part.inline_prefix[i] = prefix[first + i] - prefix[first];
@@ -346,6 +446,7 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
     }
     DecodeBatch batch;
     batch.n_jobs = uint32_t(n_items);
+    batch.blockwise = 0;
     batch.total_blocks = uint32_t(total);
     if (uint32_t(n_items) <= kInlineJobs) {
         // a short list travels in the launch parameters: no copy, no scratch
@@ -383,6 +484,18 @@ enec_status enec_compress_with_params(const void* d_in, enec_dtype dt, size_t co
 size_t enec_max_compressed_size_ranked(enec_dtype dt, size_t count) {
     const size_t base = enec_max_compressed_size(dt, count);
     return base ? base + kRankTableBytes : 0;
+}
+
+size_t enec_max_compressed_size_blockwise(enec_dtype dt, size_t count) { return max_size_blockwise(dt, count); }
+
+enec_status enec_compress_blockwise(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,
+                                    size_t* d_out_size, int* d_status, enec_stream_t stream) {
+    return compress_blockwise(d_in, dt, count, d_out, out_capacity, d_out_size, d_status, stream);
+}
+
+enec_status enec_decompress_blockwise(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
+                                      int* d_status, enec_stream_t stream) {
+    return decompress_one(d_in, in_size, dt, count, d_out, d_status, stream, false, true);
 }
 
 enec_status enec_compress_ranked(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,

@@ -21,7 +21,8 @@ struct alignas(16) Header {
     uint32_t magic;         //  0
     uint16_t version;       //  4
     uint8_t dtype;          //  6
-    uint8_t variant;        //  7: 0 = linear transform (Sec. 5.3), 1 = frequency ranks (Sec. 4.2, Algorithm 1)
+    uint8_t variant;        //  7: 0 = linear transform (Sec. 5.3), 1 = frequency ranks (Sec. 4.2, Algorithm 1),
+                            //     2 = linear transform with parameters per block (block table)
     uint64_t count;         //  8
     uint32_t block;         // 16
     uint8_t b, n, m, L;     // 20..23

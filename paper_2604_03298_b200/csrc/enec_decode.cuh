@@ -178,22 +178,50 @@ struct JobCtx {
     uint32_t a_total;
     int b, n, m;
     uint64_t off_table, off_mask, off_low, off_smhi, off_sm, off_smlo, off_high, total;
+    bool blockwise;  // parameters and offsets per block, from the block table (header byte 7 = 2)
 };
 
 // Reads and validates the header. Returns 0 or an enec_status.
 template <int DT, bool MAPPED = false>
-__device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
+__device__ inline int load_job(const DecodeJob& job, JobCtx& c, bool blockwise = false) {
     if (job.in_size < kHeaderBytes + 16) return ENEC_ERR_BAD_STREAM;
     const Header h = *reinterpret_cast<const Header*>(job.in);
     if (h.magic != kMagic || h.version != kVersion || h.dtype != DT || h.count != job.count ||
         h.block != kBlockElems || h.L != kGroupElems)
         return ENEC_ERR_BAD_STREAM;
     constexpr int E = exp_bits(DT);
-    if (h.n < 1 || h.n > E || h.m < 1 || h.m > h.n || h.b >= (1 << E) || h.variant != (MAPPED ? 1 : 0)) return ENEC_ERR_BAD_STREAM;
+    if (h.variant != (blockwise ? 2 : MAPPED ? 1 : 0)) return ENEC_ERR_BAD_STREAM;
+    if (blockwise ? (h.b | h.n | h.m) != 0 : (h.n < 1 || h.n > E || h.m < 1 || h.m > h.n || h.b >= (1 << E)))
+        return ENEC_ERR_BAD_STREAM;
     const Geometry g = make_geometry(job.count);
     if (h.nblocks != g.nblocks || h.total_groups != g.total_groups || h.a_total > g.total_groups)
         return ENEC_ERR_BAD_STREAM;
-    const Sections s = make_sections(DT, job.count, g, h.n, h.m, h.a_total, MAPPED);
+    Sections s;
+    if (blockwise) {
+        // the block table's last entry holds the sums that fix the sizes of the two variable sections
+        const uint64_t table_bytes = 16 * (uint64_t(g.nblocks) + 1);
+        if (job.in_size < kHeaderBytes + table_bytes) return ENEC_ERR_BAD_STREAM;
+        const uint4 totals = *reinterpret_cast<const uint4*>(job.in + kHeaderBytes + 16 * uint64_t(g.nblocks));
+        uint64_t low_bytes = 0;
+        if (g.nblocks) {
+            const uint32_t m_tail = (*reinterpret_cast<const uint32_t*>(job.in + kHeaderBytes + 16 * uint64_t(g.nblocks - 1)) >> 16) & 0xFFu;
+            if (totals.y < m_tail || totals.y > 8ull * g.nblocks) return ENEC_ERR_BAD_STREAM;
+            low_bytes = uint64_t(totals.y - m_tail) * (kBlockElems / 8) + uint64_t(g.tail_padded) * m_tail / 8;
+        }
+        const uint64_t high_bytes = uint64_t(totals.z) | (uint64_t(totals.w) << 32);
+        if (totals.x != 0 || high_bytes > uint64_t(g.total_groups) * 14) return ENEC_ERR_BAD_STREAM;
+        s.unmap = kHeaderBytes;
+        s.table = kHeaderBytes;
+        s.mask = s.table + align16(table_bytes);
+        s.low = s.mask + align16((uint64_t(g.total_groups) + 7) / 8);
+        s.smhi = s.low + align16(low_bytes);
+        s.sm = s.smhi + (DT == ENEC_FP16 ? align16(g.padded_count * 3 / 8) : 0);
+        s.smlo = s.sm + align16(job.count);
+        s.high = s.smlo + (DT == ENEC_FP32 ? align16(job.count * 2) : 0);
+        s.total = s.high + align16(high_bytes);
+    } else {
+        s = make_sections(DT, job.count, g, h.n, h.m, h.a_total, MAPPED);
+    }
     if (h.total_bytes != s.total || job.in_size < s.total) return ENEC_ERR_BAD_STREAM;
     c.in = job.in;
     c.out = job.out;
@@ -204,6 +232,7 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c) {
     c.b = h.b; c.n = h.n; c.m = h.m;
     c.off_table = s.table; c.off_mask = s.mask; c.off_low = s.low; c.off_smhi = s.smhi; c.off_sm = s.sm;
     c.off_smlo = s.smlo; c.off_high = s.high; c.total = s.total;
+    c.blockwise = blockwise;
     return 0;
 }
 
@@ -610,6 +639,7 @@ struct DecodeBatch {
     const uint32_t* prefix;   // device array [n_jobs + 1]: blocks before each tensor (null with jobs)
     uint32_t n_jobs;
     uint32_t total_blocks;
+    uint32_t blockwise;       // the streams are of the block-wise variant (one tensor only)
     DecodeJob inline_jobs[kInlineJobs];          // used when jobs is null (one tensor, or a short list)
     uint32_t inline_prefix[kInlineJobs + 1];
 };
@@ -702,7 +732,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
         for (uint32_t q = threadIdx.x; q < batch.n_jobs; q += blockDim.x) {
             if (all_jobs[q].count == 0) {
                 JobCtx jc;
-                const int err = load_job<DT, MAPPED>(all_jobs[q], jc);
+                const int err = load_job<DT, MAPPED>(all_jobs[q], jc, batch.blockwise != 0);
                 if (err) report(status, err);
             }
         }
@@ -759,7 +789,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                     e0 = tb[k];
                     e1 = tb[k + 1];
                 }
-                const int err = early ? load_job<DT, MAPPED>(job, jc) : ENEC_ERR_BAD_STREAM;
+                const int err = early ? load_job<DT, MAPPED>(job, jc, batch.blockwise != 0) : ENEC_ERR_BAD_STREAM;
                 if (err) {
                     *abort_flag = 1;
                     report(status, err);
@@ -785,19 +815,46 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             const bool tail = (k + 1 == jc.nblocks);
             const uint32_t N = tail ? jc.tail_padded : kBlockElems;
             const uint32_t real = tail ? jc.tail_real : kBlockElems;
-            if (t1 < t0 || t1 - t0 > (N >> 4) || t1 > jc.a_total) {
+            int blk_b = jc.b, blk_n = jc.n, blk_m = jc.m;
+            uint64_t low_src = jc.off_low + uint64_t(k) * (kBlockElems / 8) * uint32_t(jc.m);
+            uint64_t h0;
+            uint32_t expect;
+            bool sound;
+            if (jc.blockwise) {
+                // this block's parameters and offsets, and the next entry for the end of its records
+                const uint4 own = *reinterpret_cast<const uint4*>(jc.in + kHeaderBytes + 16 * uint64_t(k));
+                const uint4 nxt = *reinterpret_cast<const uint4*>(jc.in + kHeaderBytes + 16 * uint64_t(k + 1));
+                blk_b = int(own.x & 0xFFu); blk_n = int((own.x >> 8) & 0xFFu); blk_m = int((own.x >> 16) & 0xFFu);
+                sound = blk_n >= 1 && blk_n <= exp_bits(DT) && blk_m >= 1 && blk_m <= blk_n && blk_b < (1 << exp_bits(DT)) &&
+                        (own.x >> 24) == 0;
+                hbits = sound ? blk_n - blk_m : 0;
+                if (sound) L = make_stage_layout(DT, blk_m, hbits, false);
+                const uint64_t rec0 = uint64_t(own.z) | (uint64_t(own.w) << 32), rec1 = uint64_t(nxt.z) | (uint64_t(nxt.w) << 32);
+                const uint64_t rec_size = 2 * uint64_t(hbits);
+                sound = sound && (k != 0 || (own.y == 0 && rec0 == 0));  // the sums start at zero
+                sound = sound && rec1 >= rec0 && rec1 <= jc.total - jc.off_high && nxt.y == own.y + uint32_t(blk_m) &&
+                        (rec_size ? (rec1 - rec0) % rec_size == 0 : rec1 == rec0);
+                expect = sound && rec_size ? uint32_t((rec1 - rec0) / rec_size) : 0;
+                low_src = jc.off_low + uint64_t(own.y) * (kBlockElems / 8);
+                sound = sound && expect <= (N >> 4) && low_src + uint64_t(N) * uint32_t(blk_m) / 8 <= jc.off_smhi;
+                h0 = jc.off_high + rec0;
+            } else {
+                sound = t1 >= t0 && t1 - t0 <= (N >> 4) && t1 <= jc.a_total;
+                expect = t1 - t0;
+                h0 = jc.off_high + uint64_t(t0) * (2 * hbits);
+            }
+            if (!sound) {
                 *abort_flag = 1;
                 report(status, ENEC_ERR_BAD_STREAM);
                 failed = true;
                 break;
             }
-            const uint64_t h0 = jc.off_high + uint64_t(t0) * (2 * hbits);
             const uint64_t w0 = h0 & ~uint64_t(15);
-            uint32_t staged = t1 - t0 < L.cap ? t1 - t0 : L.cap;  // records staged in shared memory
+            uint32_t staged = expect < L.cap ? expect : L.cap;  // records staged in shared memory
             if (hbits == 0) staged = 0;
             const uint64_t w1 = align16(h0 + uint64_t(staged) * (2 * hbits));
             const uint32_t mask_bytes = uint32_t(align16(((N >> 4) + 7) / 8));
-            const uint32_t low_bytes = uint32_t(align16(uint64_t(N) * jc.m / 8));
+            const uint32_t low_bytes = uint32_t(align16(uint64_t(N) * uint32_t(blk_m) / 8));
             const uint32_t smhi_bytes = DT == ENEC_FP16 ? uint32_t(align16(uint64_t(N) * 3 / 8)) : 0;
             const uint32_t sm_bytes = uint32_t(align16(real));
             const uint32_t raw_bytes = staged ? uint32_t(w1 - w0) : 0;
@@ -805,12 +862,12 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             BlockDesc* d = reinterpret_cast<BlockDesc*>(st);
             d->first = uint32_t(h0 - w0);
             d->staged = staged;
-            d->expect = t1 - t0;
+            d->expect = expect;
             d->N = N;
             d->real = real;
-            d->code = uint32_t(jc.m * 8 + hbits);
-            d->b = uint32_t(jc.b);
-            d->n = uint32_t(jc.n);
+            d->code = uint32_t(blk_m * 8 + hbits);
+            d->b = uint32_t(blk_b);
+            d->n = uint32_t(blk_n);
             d->L = L;
             d->out = jc.out + uint64_t(k) * kBlockElems * (DT == ENEC_FP32 ? 2 : 1);
             if (DT == ENEC_FP32) {
@@ -827,12 +884,12 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                                               (MAPPED ? kRankTableBytes : 0u));
             if constexpr (MAPPED) bulk_g2s(st + kStageRankTable, jc.in + kHeaderBytes, kRankTableBytes, &ctl->full[s]);
             bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
-            bulk_g2s(st + L.low, jc.in + jc.off_low + uint64_t(k) * (kBlockElems / 8) * jc.m, low_bytes, &ctl->full[s]);
+            bulk_g2s(st + L.low, jc.in + low_src, low_bytes, &ctl->full[s]);
             if (DT == ENEC_FP16)
                 bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
             bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
             if (raw_bytes) bulk_g2s(st + L.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
-            if (k + 2 <= jc.nblocks) t2 = table[k + 2];  // for the tensor's next block
+            if (!jc.blockwise && k + 2 <= jc.nblocks) t2 = table[k + 2];  // for the tensor's next block
         }
         if (failed) {
             if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }

@@ -158,17 +158,19 @@ __device__ __forceinline__ int choose_m(const unsigned long long (&width_count)[
     return best_m;
 }
 
-// Sec. 5.5 phases 2 and 3 on the finished histogram; all kHistThreads threads of one CTA.
+// Sec. 5.5 phases 2 and 3 on a finished histogram; threads 0..255 of one CTA, thread t bringing the count of
+// exponent t (`mine`; zero beyond the field; at least one count is non-zero). All of them return with the same
+// (b, n, m). Every thread of the CTA must call it (it synchronises the CTA).
 template <int DT>
-__device__ void parameter_search(EncodeControl* ctl) {
+__device__ void parameter_search_counts(unsigned long long mine, int& out_b, int& out_n, int& out_m) {
     constexpr int E = HistShape<DT>::E;
     constexpr int kBins = 1 << E;
     __shared__ unsigned long long s_hist[256];
     __shared__ unsigned long long s_key[kHistThreads / 32];
     __shared__ unsigned long long s_width_count[9];
-    __shared__ int s_lo, s_hi, s_b, s_n;
+    __shared__ int s_lo, s_hi, s_b, s_n, s_m;
     const uint32_t tid = threadIdx.x;
-    s_hist[tid] = tid < uint32_t(kBins) ? ld_relaxed_u64(&ctl->hist[tid]) : 0ull;
+    s_hist[tid] = tid < uint32_t(kBins) ? mine : 0ull;
     if (tid < 9) s_width_count[tid] = 0;
     if (tid == 0) { s_lo = kBins; s_hi = -1; }
     __syncthreads();
@@ -206,10 +208,24 @@ __device__ void parameter_search(EncodeControl* ctl) {
         atomicAdd(&s_width_count[bit_width_u32(y)], s_hist[tid]);
     }
     __syncthreads();
+    if (tid == 0) s_m = choose_m(s_width_count, n);
+    __syncthreads();
+    out_b = b;
+    out_n = n;
+    out_m = s_m;
+    __syncthreads();  // the shared words may be written again by the next call
+}
+
+// The search on a tensor's histogram in its control words; the result goes back there.
+template <int DT>
+__device__ void parameter_search(EncodeControl* ctl) {
+    const uint32_t tid = threadIdx.x;
+    int b, n, m;
+    parameter_search_counts<DT>(tid < uint32_t(1 << HistShape<DT>::E) ? ld_relaxed_u64(&ctl->hist[tid]) : 0ull, b, n, m);
     if (tid == 0) {
         ctl->b = b;
         ctl->n = n;
-        ctl->m = choose_m(s_width_count, n);
+        ctl->m = m;
     }
 }
 
@@ -1278,16 +1294,17 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
     }
 }
 
-// Stream of an empty tensor: header, (frequency-rank variant: an all-zero rank table) and a one-entry table.
+// Stream of an empty tensor: header, (frequency-rank variant: an all-zero rank table) and a one-entry table
+// (16 zero bytes in every variant).
 __global__ void enec_encode_empty_kernel(uint8_t* out, int dt, int b, int n, int m, unsigned long long* out_size,
-                                         int ranked = 0) {
+                                         int variant = 0) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    const uint32_t table_at = kHeaderBytes + (ranked ? kRankTableBytes : 0);
+    const uint32_t table_at = kHeaderBytes + (variant == 1 ? kRankTableBytes : 0);
     Header hd;
     hd.magic = kMagic;
     hd.version = kVersion;
     hd.dtype = uint8_t(dt);
-    hd.variant = ranked ? 1 : 0;
+    hd.variant = uint8_t(variant);
     hd.count = 0;
     hd.block = kBlockElems;
     hd.b = uint8_t(b); hd.n = uint8_t(n); hd.m = uint8_t(m); hd.L = kGroupElems;

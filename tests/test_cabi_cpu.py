@@ -24,7 +24,8 @@ def declared_functions():
 def test_header_declares_the_expected_entry_points():
     names = declared_functions()
     for want in ("enec_max_compressed_size", "enec_compress", "enec_compress_with_params", "enec_decompress",
-                 "enec_compress_batched", "enec_decompress_batched", "enec_compress_noalloc", "enec_launch_count", "enec_allocation_count",
+                 "enec_compress_batched", "enec_decompress_batched", "enec_compress_noalloc", "enec_compress_blockwise",
+                 "enec_decompress_blockwise", "enec_max_compressed_size_blockwise", "enec_launch_count", "enec_allocation_count",
                  "enec_version"):
         assert want in names
 
@@ -41,6 +42,13 @@ def test_max_compressed_size_matches_oracle(libenec, oracle):
     for dt in (0, 1, 2):
         for count in (0, 1, 15, 16, 17, 4096, 16383, 16384, 16385, 123457, 1 << 20, 128256 * 4096, (1 << 36) - 1):
             assert f(dt, count) == oracle.max_compressed_size(dt, count)
+    assert f(3, 100) == 0 and f(0, 1 << 36) == 0
+    f = libenec.enec_max_compressed_size_blockwise
+    f.argtypes = [ctypes.c_int, ctypes.c_size_t]
+    f.restype = ctypes.c_size_t
+    for dt in (0, 1, 2):
+        for count in (0, 1, 15, 16, 17, 4096, 16383, 16384, 16385, 123457, 1 << 20, 128256 * 4096, (1 << 36) - 1):
+            assert f(dt, count) == oracle.max_compressed_size_blockwise(dt, count)
     assert f(3, 100) == 0 and f(0, 1 << 36) == 0
 
 
