@@ -469,6 +469,66 @@ def run_ours(args):
     barrier()
     ms_comp_ranked = runner.max_over_ranks(sum(e[0].elapsed_time(e[1]) for e in ev3) / args.steps)
     ms_dec_ranked = runner.max_over_ranks(sum(e[1].elapsed_time(e[2]) for e in ev3) / args.steps)
+    # ablation: parameters per block (Sec. 5.5 on every block's own histogram), same steps, one stream
+    for _ in range(2):
+        cs.compress_all(blockwise=True)
+        cs.decompress_all(blockwise=True)
+    torch.cuda.synchronize()
+    cs.check_status()
+    cs.verify_roundtrip()
+    blockwise_bytes = runner.sum_over_ranks(cs.compressed_bytes())
+    ev4 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    for k in range(args.steps):
+        ev4[k][0].record()
+        cs.compress_all(blockwise=True)
+        ev4[k][1].record()
+        cs.decompress_all(blockwise=True)
+        ev4[k][2].record()
+    barrier()
+    ms_comp_blockwise = runner.max_over_ranks(sum(e[0].elapsed_time(e[1]) for e in ev4) / args.steps)
+    ms_dec_blockwise = runner.max_over_ranks(sum(e[1].elapsed_time(e[2]) for e in ev4) / args.steps)
+
+    # the same comparison on two side sets where parameters per block could matter: the heavy-tailed stress set
+    # (a sample of it) and one Gaussian decoder layer with the generator's exact zeros left in
+    def per_block_side_set(side_specs, keep_zeros):
+        side_raw = [synth.make_tensor(sp, "cuda", keep_zeros=keep_zeros) for sp in side_specs]
+        side = runner.CodecSet.allocate(side_raw)
+        res = {"raw_bytes": side.raw_bytes, "tensors": len(side_raw)}
+        for name, kw in (("per_tensor", {}), ("per_block", {"blockwise": True})):
+            for _ in range(3):
+                side.compress_all(**kw)
+                side.decompress_all(**kw)
+            torch.cuda.synchronize()
+            side.check_status()
+            side.verify_roundtrip()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            reps = 5
+            e[0].record()
+            for _ in range(reps):
+                side.compress_all(**kw)
+            e[1].record()
+            for _ in range(reps):
+                side.decompress_all(**kw)
+            e[2].record()
+            torch.cuda.synchronize()
+            res[name] = {"compression_ratio": side.raw_bytes / side.compressed_bytes(),
+                         "compress_gbs": side.raw_bytes * reps / (e[0].elapsed_time(e[1]) * 1e-3) / 1e9,
+                         "decompress_gbs": side.raw_bytes * reps / (e[1].elapsed_time(e[2]) * 1e-3) / 1e9}
+        return res
+
+    per_block_sides = None
+    if rank == 0:
+        heavy = synth.config_specs(4)
+        per_block_sides = {
+            "heavy_tailed_sample": dict(per_block_side_set(heavy[:8] + heavy[32:40] + heavy[64:72] + heavy[96:104], False),
+                                        sample="sample: 32 of the 128 tensors of the heavy-tailed stress set (8 each of "
+                                               "fp16 Laplace, fp16 Student-t, bf16 Laplace, bf16 Student-t)"),
+            "gaussian_layer_zeros_kept": dict(per_block_side_set(synth.config_specs(2), True),
+                                              sample="one Llama-3-8B-shaped bf16 decoder layer, the normal generator's "
+                                                     "exact zeros left in"),
+        }
+
     cs.compress_all()      # back to the linear streams for what follows
     torch.cuda.synchronize()
     cs.check_status()
@@ -585,6 +645,14 @@ def run_ours(args):
                              "note": "same tensors through enec_compress_batched (one call per dtype of the set)"},
         "compression_ratio": total_raw / total_comp,
         "compression_ratio_zeros_kept": zeros_kept,
+        "ablation_per_block": {
+            "compression_ratio": total_raw / blockwise_bytes,
+            "decompress": {"value": total_raw / (ms_dec_blockwise * 1e-3) / 1e9, "unit": "GB/s"},
+            "compress": {"value": total_raw / (ms_comp_blockwise * 1e-3) / 1e9, "unit": "GB/s"},
+            "side_sets": per_block_sides,
+            "note": "enec_compress_blockwise / enec_decompress_blockwise tensor by tensor on one stream: the search of "
+                    "Sec. 5.5 on every 16384-element block's own histogram, a 16-byte table entry per block; compare "
+                    "compression_ratio and the one-stream rates of this workload"},
         "ablation_frequency_ranks": {
             "compression_ratio": total_raw / ranked_bytes,
             "decompress": {"value": total_raw / (ms_dec_ranked * 1e-3) / 1e9, "unit": "GB/s"},

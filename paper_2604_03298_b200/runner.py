@@ -59,8 +59,11 @@ class CodecSet:
     def allocate(cls, raw: List[torch.Tensor], share_output: bool = False) -> "CodecSet":
         dev = raw[0].device
         cs = cls(raw=[t.contiguous() for t in raw])
-        # room for either variant of the stream (the frequency-rank variant is 256 bytes longer)
-        cs.streams = [torch.empty(enec.enec_max_compressed_size_ranked(_DT[t.dtype], t.numel()), dtype=torch.uint8, device=dev)
+        # room for every variant of the stream (the frequency-rank variant is 256 bytes longer, the block-wise one
+        # has the larger table)
+        cs.streams = [torch.empty(max(enec.enec_max_compressed_size_ranked(_DT[t.dtype], t.numel()),
+                                      enec.enec_max_compressed_size_blockwise(_DT[t.dtype], t.numel())),
+                                  dtype=torch.uint8, device=dev)
                       for t in cs.raw]
         cs.shared_outs = share_output
         if share_output:
@@ -105,15 +108,19 @@ class CodecSet:
             done.record(s)
             main.wait_event(done)
 
-    def compress_all(self, params=None, n_streams: int = 1, ranked: bool = False) -> None:
+    def compress_all(self, params=None, n_streams: int = 1, ranked: bool = False, blockwise: bool = False) -> None:
         """One enec_compress per tensor (no host synchronisation), on the current stream or spread over
-        n_streams side streams. ranked: the frequency-rank variant (enec_compress_ranked) instead."""
-        self.spread(n_streams, lambda i: self._compress_one(i, params, ranked))
+        n_streams side streams. ranked: the frequency-rank variant (enec_compress_ranked) instead; blockwise: the
+        variant with parameters per block (enec_compress_blockwise)."""
+        self.spread(n_streams, lambda i: self._compress_one(i, params, ranked, blockwise))
 
-    def _compress_one(self, i: int, params, ranked: bool = False) -> None:
+    def _compress_one(self, i: int, params, ranked: bool = False, blockwise: bool = False) -> None:
         t = self.raw[i]
         dt = _DT[t.dtype]
-        if ranked:
+        if blockwise:
+            st = enec.enec_compress_blockwise(t, dt, t.numel(), self.streams[i], self.streams[i].numel(),
+                                              self.sizes[i:i + 1], self.status)
+        elif ranked:
             st = enec.enec_compress_ranked(t, dt, t.numel(), self.streams[i], self.streams[i].numel(),
                                            self.sizes[i:i + 1], self.status)
         elif params is None:
@@ -125,15 +132,15 @@ class CodecSet:
         if st != 0:
             raise enec.EnecError(st, f"enec_compress tensor {i}")
 
-    def decompress_all(self, n_streams: int = 1, ranked: bool = False) -> None:
+    def decompress_all(self, n_streams: int = 1, ranked: bool = False, blockwise: bool = False) -> None:
         """One enec_decompress per tensor, on the current stream or spread over n_streams side streams. The
         stream length passed is the buffer's capacity; the true length is in the stream header and is checked
         against it on the device."""
-        self.spread(n_streams, lambda i: self._decompress_one(i, ranked))
+        self.spread(n_streams, lambda i: self._decompress_one(i, ranked, blockwise))
 
-    def _decompress_one(self, i: int, ranked: bool = False) -> None:
+    def _decompress_one(self, i: int, ranked: bool = False, blockwise: bool = False) -> None:
         t = self.raw[i]
-        fn = enec.enec_decompress_ranked if ranked else enec.enec_decompress
+        fn = enec.enec_decompress_blockwise if blockwise else enec.enec_decompress_ranked if ranked else enec.enec_decompress
         st = fn(self.streams[i], self.streams[i].numel(), _DT[t.dtype], t.numel(),
                                   self.outs[i], self.status)
         if st != 0:
