@@ -429,8 +429,10 @@ __device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, ui
 // run. bf16 with n < 8 uses it only when b + 2^(n-1) <= 255: then x = (b + 2^(n-1)) - (y ^ 2^(n-1)) never
 // borrows across bytes for a stream that came from real data (x is a field value), and a plain
 // subtraction serves; other bf16 tensors with n < 8 take the general body.
+// The frequency-rank variant (MAPPED) has no sign position: nothing is flipped, the slot of narrow groups holds
+// zeros, and the exponent comes from the stage's rank table (shared address in r.c4) instead of the subtraction.
 // tid = 0..255; thread tid owns the runs c * 2048 + 8 tid (c < 8).
-template <int DT, int M, int HB>
+template <int DT, int M, int HB, bool MAPPED = false>
 __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_low, uint32_t s_smhi, uint32_t tid) {
     constexpr int n = M + HB;
     constexpr uint32_t Hm = 0x80808080u;
@@ -474,12 +476,15 @@ __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_lo
             if constexpr (HB > 0) {
                 v.x += hi[q].x << M;  // disjoint bits
                 v.y += hi[q].y << M;
-            } else {
+            } else if constexpr (!MAPPED) {
                 v.x ^= r.s4;
                 v.y ^= r.s4;
             }
             uint32_t x0, x1;
-            if constexpr (DT == ENEC_FP16) {
+            if constexpr (MAPPED) {
+                x0 = table4(r.c4, v.x);
+                x1 = table4(r.c4, v.y);
+            } else if constexpr (DT == ENEC_FP16) {
                 // b + 2^(n-1) < 128: the guard bit absorbs any borrow and is masked away with the field
                 x0 = r.c4_or_h - v.x;
                 x1 = r.c4_or_h - v.y;
@@ -922,12 +927,11 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                        o_exp = d->L.expanded;
         const uint32_t sbit = 1u << (n - 1);
         const bool simple_sub = DT == ENEC_FP16 || n == 8 || b + sbit <= 255;
-        // ranks go through the general body: the branch-free one is built on the subtraction
-        const bool full_block = !MAPPED && N == kBlockElems && d->real == kBlockElems && expect <= cap && simple_sub;
+        const bool full_block = N == kBlockElems && d->real == kBlockElems && expect <= cap && (MAPPED || simple_sub);
         // preparation: ranks of the wide groups and expanded records
         if (hbits > 0) {
             // the branch-free body wants narrow groups to point at the flip slot and flipped records
-            const uint32_t flip4 = rep4(1u << (hbits - 1));
+            const uint32_t flip4 = MAPPED ? 0u : rep4(1u << (hbits - 1));
             if (tid == 0) sts128(st + o_exp + cap * 16, make_uint4(flip4, flip4, flip4, flip4));
             const uint32_t wide = build_rank_array(st + d->L.mask, st + o_rank, N, tid, full_block ? cap : kNotWide);
             if (wide != expect && lane == 0) {  // the prefix table must agree with the mask
@@ -959,18 +963,16 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
         switch (code) {
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
-        if constexpr (MAPPED) decode_block<DTV, MV, HV, true>(r, st + o_low, st + o_smhi, N, tid); \
-        else if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid); \
-        else decode_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, N, tid);                  \
+        if (full_block) decode_full_block<DTV, MV, HV, MAPPED>(r, st + o_low, st + o_smhi, tid); \
+        else decode_block<DTV, MV, HV, MAPPED>(r, st + o_low, st + o_smhi, N, tid);          \
         break;
             ENEC_FOR_EACH_MH(ENEC_CASE, DT)
 #undef ENEC_CASE
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
         if constexpr (DTV != ENEC_FP16) {                                                    \
-            if constexpr (MAPPED) decode_block<DTV, MV, HV, true>(r, st + o_low, st + o_smhi, N, tid); \
-            else if (full_block) decode_full_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, tid); \
-            else decode_block<DTV, MV, HV>(r, st + o_low, st + o_smhi, N, tid);              \
+            if (full_block) decode_full_block<DTV, MV, HV, MAPPED>(r, st + o_low, st + o_smhi, tid); \
+            else decode_block<DTV, MV, HV, MAPPED>(r, st + o_low, st + o_smhi, N, tid);      \
         }                                                                                    \
         break;
             ENEC_FOR_EACH_MH_BF16_ONLY(ENEC_CASE, DT)
