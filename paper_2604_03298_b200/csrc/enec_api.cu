@@ -3,6 +3,7 @@
 #include <map>
 #include <mutex>
 #include <utility>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -21,6 +22,7 @@ struct DeviceInfo {
     bool encode_attr_set[3] = {false, false, false};
     bool batch_attr_set[3] = {false, false, false};
     bool blockwise_attr_set[3] = {false, false, false};
+    bool split_attr_set[3] = {false, false, false};
 };
 
 // Per-device facts, for device ordinals below kMaxDevices (null beyond: the caller fails with ENEC_ERR_CUDA).
@@ -108,9 +110,51 @@ static void place_job(EncodeJob& job, uint8_t* scratch, uint32_t epoch) {
     job.epoch = epoch;
 }
 
+// Tensors of split_min_blocks() .. split_max_blocks() - 1 blocks are compressed in the split form (pack kernel, then
+// the kernel that places the records). Below that range the third launch costs more than the look-back it replaces;
+// above it every CTA has so many blocks that the look-back no longer shows. ENEC_SPLIT_MIN_BLOCKS and
+// ENEC_SPLIT_MAX_BLOCKS in the environment override the bounds (read once; for measurements and tests).
+static uint32_t env_blocks(const char* name, uint32_t fallback) {
+    const char* e = getenv(name);
+    return e && *e ? uint32_t(strtoul(e, nullptr, 10)) : fallback;
+}
+static uint32_t split_min_blocks() {
+    static const uint32_t value = env_blocks("ENEC_SPLIT_MIN_BLOCKS", 2048u);
+    return value;
+}
+static uint32_t split_max_blocks() {
+    static const uint32_t value = env_blocks("ENEC_SPLIT_MAX_BLOCKS", 24576u);
+    return value;
+}
+
+template <int DT>
+static enec_status launch_split(const EncodeJob& job, uint32_t nblocks, int* d_status, DeviceInfo& info,
+                                cudaStream_t stream) {
+    if (!info.split_attr_set[DT]) {
+        if (cudaFuncSetAttribute(enec_pack_tensor_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(kPackSmemBytes)) != cudaSuccess ||
+            cudaFuncSetAttribute(enec_place_records_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(kPlaceSmemBytes)) != cudaSuccess)
+            return ENEC_ERR_CUDA;
+        info.split_attr_set[DT] = true;
+    }
+    uint32_t grid = uint32_t(info.sms) * 4;
+    if (grid > nblocks) grid = nblocks;
+    if (launch_pdl(enec_pack_tensor_kernel<DT>, grid, kPackThreads, kPackSmemBytes, stream, job, d_status) != cudaSuccess)
+        return ENEC_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    grid = uint32_t(info.sms) * 2;
+    if (grid > nblocks) grid = nblocks;
+    if (grid > kPlaceMaxCtas) grid = kPlaceMaxCtas;
+    if (launch_pdl(enec_place_records_kernel<DT>, grid, kPlaceThreads, kPlaceSmemBytes, stream, job, d_status) != cudaSuccess)
+        return ENEC_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ENEC_OK;
+}
+
 template <int DT>
 static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool search, int* d_status, DeviceInfo& info,
-                                 cudaStream_t stream) {
+                                 cudaStream_t stream, bool may_split = false) {
     if (search) {
         const uint32_t smem = HistShape<DT>::kBytes;
         if (!info.hist_attr_set[DT]) {
@@ -132,6 +176,7 @@ static enec_status launch_encode(const EncodeJob& job, uint32_t nblocks, bool se
                                     job.count, job.ctl);
         if (herr != cudaSuccess) return ENEC_ERR_CUDA;
         g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (may_split && !job.ranked && nblocks >= split_min_blocks() && nblocks < split_max_blocks()) return launch_split<DT>(job, nblocks, d_status, info, stream);
     }
     if (!info.encode_attr_set[DT]) {
         if (cudaFuncSetAttribute(enec_encode_kernel<DT, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -205,7 +250,8 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
     if (!found) return ENEC_ERR_CUDA;
     DeviceInfo& info = *found;
     const Geometry g = make_geometry(count);
-    const size_t need = kControlBytes + size_t(g.nblocks) * sizeof(unsigned long long);
+    // control words, a state word per block, and the progress words of the kernel that places the records
+    const size_t need = kControlBytes + (size_t(g.nblocks) + kPlaceMaxCtas) * sizeof(unsigned long long);
     // the scratch area carries state from call to call, which a replayed recording would not see
     cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return ENEC_ERR_CUDA;
@@ -224,9 +270,9 @@ static enec_status compress_common(const void* d_in, enec_dtype dt, size_t count
     job.from_search = with_params ? 0 : 1;
     job.check = with_params ? 1 : 0;
     job.ranked = ranked ? 1 : 0;
-    st = dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream)
-         : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream)
-                           : launch_encode<ENEC_FP32>(job, g.nblocks, !with_params, d_status, info, stream);
+    st = dt == ENEC_BF16   ? launch_encode<ENEC_BF16>(job, g.nblocks, !with_params, d_status, info, stream, true)
+         : dt == ENEC_FP16 ? launch_encode<ENEC_FP16>(job, g.nblocks, !with_params, d_status, info, stream, true)
+                           : launch_encode<ENEC_FP32>(job, g.nblocks, !with_params, d_status, info, stream, true);
     if (st != ENEC_OK) mark_compress_scratch_unclean(dev, stream);  // a kernel of the call may not have run
     return st;
 }

@@ -15,7 +15,7 @@
 // The input is read twice, as by enec_compress (histogram pass, encode pass).
 #pragma once
 
-#include "enec_encode.cuh"
+#include "enec_pack.cuh"
 
 namespace enec {
 
@@ -49,31 +49,7 @@ struct BlockwiseJob {
     unsigned long long* out_size;  // device, may be null
 };
 
-constexpr int kBlockwiseThreads = 256;
-
-__device__ __forceinline__ TransformCtx make_transform_ctx(int dt_exp_bits, int b, int n) {
-    TransformCtx tc;
-    tc.b4 = rep4(uint32_t(b));
-    tc.b4_or_h = tc.b4 | 0x80808080u;
-    tc.nmask4 = rep4((1u << n) - 1);
-    tc.s4 = rep4(1u << (n - 1));
-    tc.emask4 = rep4((1u << dt_exp_bits) - 1);
-    tc.n = n;
-    tc.E = dt_exp_bits;
-    tc.lut = 0;
-    return tc;
-}
-
-// Exponent field of element i of a block at `in_bytes`, and the 16-bit word that carries it (for fp32 the high half).
-template <int DT>
-__device__ __forceinline__ uint32_t exponent_word(const uint8_t* in_bytes, uint32_t i) {
-    return DT == ENEC_FP32 ? reinterpret_cast<const uint32_t*>(in_bytes)[i] >> 16
-                           : uint32_t(reinterpret_cast<const uint16_t*>(in_bytes)[i]);
-}
-template <int DT>
-__device__ __forceinline__ uint32_t exponent_of_word(uint32_t w) {
-    return DT != ENEC_FP16 ? (w >> 7) & 0xFFu : (w >> 10) & 0x1Fu;
-}
+constexpr int kBlockwiseThreads = kPackThreads;
 
 // The block table's entries hold each block's own m and record bytes: turn them into sums over the blocks
 // before, append the totals and write the header. All threads of one CTA, after every entry is visible.
@@ -273,128 +249,24 @@ enec_block_params_kernel(const BlockwiseJob job, int* status) {
     (void)status;
 }
 
-// A tensor's last block when it is not full (N padded elements, N a power of two up to 16384, `real` present), all
-// 256 threads, element by element and bit by bit (Algorithm 2 followed for every set bit). `work` is shared memory:
-// mask [32 words] | low plane [16384 bytes; the fp16 plane 10240 bytes in, behind a low plane of m <= 5] | records.
-template <int DT>
-__device__ __forceinline__ uint32_t tail_word(const uint8_t* in_bytes, uint32_t i) {
-    return DT == ENEC_FP32 ? reinterpret_cast<const uint32_t*>(in_bytes)[i] >> 16
-                           : uint32_t(reinterpret_cast<const uint16_t*>(in_bytes)[i]);
-}
-
-constexpr uint32_t kTailWorkWords = 32 + kBlockElems / 4 + kGroupsPerBlock * 14 / 4;
-
-template <int DT>
-__device__ __noinline__ void pack_tail_block(const uint8_t* in_bytes, uint32_t N, uint32_t real, int b, int n, int m,
-                                             uint8_t* out_sm, uint8_t* out_low, uint8_t* out_smhi, uint8_t* out_mask,
-                                             uint8_t* out_smlo, uint8_t* out_rec, uint8_t* work) {
-    const uint32_t tid = threadIdx.x;
-    const uint32_t hbits = uint32_t(n - m);
-    const uint32_t groups = N >> 4;
-    const uint32_t nmask = (1u << n) - 1;
-    uint32_t* s_mask = reinterpret_cast<uint32_t*>(work);
-    uint32_t* s_low = s_mask + 32;
-    uint32_t* s_hi3 = s_low + 10240 / 4;
-    uint32_t* s_rec = s_low + kBlockElems / 4;
-    for (uint32_t i = tid; i < kTailWorkWords; i += kBlockwiseThreads) s_mask[i] = 0;
-    __syncthreads();
-    for (uint32_t i = tid; i < N; i += kBlockwiseThreads) {
-        uint32_t y = 0, hs = 0;
-        if (i < real) {
-            if (DT == ENEC_FP32)
-                reinterpret_cast<uint16_t*>(out_smlo)[i] = uint16_t(reinterpret_cast<const uint32_t*>(in_bytes)[i]);
-            const uint32_t w = tail_word<DT>(in_bytes, i);
-            y = uint32_t(b - int(exponent_of_word<DT>(w))) & nmask;
-            if (DT != ENEC_FP16) {
-                out_sm[i] = uint8_t(((w >> 8) & 0x80) | (w & 0x7F));
-            } else {
-                out_sm[i] = uint8_t(w);
-                hs = ((w >> 13) & 4) | ((w >> 8) & 3);
-            }
-        } else {
-            if (i < uint32_t(align16(real))) out_sm[i] = 0;
-            if (DT == ENEC_FP32 && 2 * i < uint32_t(align16(2 * uint64_t(real)))) reinterpret_cast<uint16_t*>(out_smlo)[i] = 0;
-        }
-        if (y >> m) atomicOr(&s_mask[i >> 9], 1u << ((i >> 4) & 31));
-        for (int q = 0; q < m; ++q)
-            if ((y >> q) & 1) {
-                uint32_t pos; int bit;
-                alg2_locate(N, m, i, q, pos, bit);
-                atomicOr(&s_low[pos >> 2], 1u << (8 * (pos & 3) + bit));
-            }
-        if (DT == ENEC_FP16)
-            for (int q = 0; q < 3; ++q)
-                if ((hs >> q) & 1) {
-                    uint32_t pos; int bit;
-                    alg2_locate(N, 3, i, q, pos, bit);
-                    atomicOr(&s_hi3[pos >> 2], 1u << (8 * (pos & 3) + bit));
-                }
-    }
-    __syncthreads();
-    if (hbits > 0) {
-        for (uint32_t i = tid; i < real; i += kBlockwiseThreads) {
-            const uint32_t grp = i >> 4;
-            if (!((s_mask[grp >> 5] >> (grp & 31)) & 1)) continue;
-            const uint32_t hv = (uint32_t(b - int(exponent_of_word<DT>(tail_word<DT>(in_bytes, i)))) & nmask) >> m;
-            if (!hv) continue;
-            uint32_t rank = __popc(s_mask[grp >> 5] & ((1u << (grp & 31)) - 1));
-            for (uint32_t wq = 0; wq < (grp >> 5); ++wq) rank += __popc(s_mask[wq]);
-            for (uint32_t q = 0; q < hbits; ++q)
-                if ((hv >> q) & 1) {
-                    uint32_t pos; int bit;
-                    alg2_locate(16, int(hbits), i & 15, int(q), pos, bit);
-                    pos += rank * 2 * hbits;
-                    atomicOr(&s_rec[pos >> 2], 1u << (8 * (pos & 3) + bit));
-                }
-        }
-    }
-    __syncthreads();
-    // planes out, padded to 16 bytes with zeros (the shared words behind them are zero)
-    for (uint32_t i = tid; i < uint32_t(align16(uint64_t(N) * m / 8)) / 4; i += kBlockwiseThreads)
-        reinterpret_cast<uint32_t*>(out_low)[i] = s_low[i];
-    for (uint32_t i = tid; i < uint32_t(align16((groups + 7) / 8)) / 4; i += kBlockwiseThreads)
-        reinterpret_cast<uint32_t*>(out_mask)[i] = s_mask[i];
-    if (DT == ENEC_FP16)
-        for (uint32_t i = tid; i < uint32_t(align16(uint64_t(N) * 3 / 8)) / 4; i += kBlockwiseThreads)
-            reinterpret_cast<uint32_t*>(out_smhi)[i] = s_hi3[i];
-    uint32_t wide_count = 0;
-    for (uint32_t wq = 0; wq < 32; ++wq) wide_count += __popc(s_mask[wq]);
-    for (uint32_t i = tid; i < wide_count * hbits; i += kBlockwiseThreads)
-        reinterpret_cast<uint16_t*>(out_rec)[i] = reinterpret_cast<const uint16_t*>(s_rec)[i];
-    __syncthreads();
-}
-
-constexpr uint32_t kPackSmemBytes = 2 * kBlockElems + 16;  // low plane (fp16 plane behind it) | wide groups' values + a spare slot
-static_assert(kTailWorkWords * 4 <= kPackSmemBytes, "the tail packer works inside the pack kernel's shared memory");
-
 // CTA c packs the blocks c, c + grid, ...; everything it needs about a block is in the block's table entry.
 template <int DT>
 __global__ void __launch_bounds__(kBlockwiseThreads, 4)
 enec_pack_blocks_kernel(const BlockwiseJob job, int* status) {
     extern __shared__ __align__(16) uint8_t pack_smem[];
     __shared__ __align__(16) uint32_t s_mask[32];
-    uint8_t* s_low = pack_smem;
-    uint8_t* s_hi3 = pack_smem + 10240;  // fp16 only (m <= 5, so the low plane ends below)
-    const uint32_t s_exp = smem_u32(pack_smem) + kBlockElems;
-    constexpr uint32_t kSpare = kGroupsPerBlock * 16;
     constexpr uint32_t kElemBytes = DT == ENEC_FP32 ? 4 : 2;
-    constexpr int E = HistShape<DT>::E;
     pdl_launch_dependents();
     pdl_wait();  // nothing above touches global memory
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const Geometry g = make_geometry(job.count);
     const BlockEntry* table = reinterpret_cast<const BlockEntry*>(job.out + kHeaderBytes);
     const BlockEntry totals = table[g.nblocks];
     const uint32_t m_tail = table[g.nblocks - 1].m;
     const uint64_t low_bytes = uint64_t(totals.m_before - m_tail) * (kBlockElems / 8) + uint64_t(g.tail_padded) * m_tail / 8;
     const Sections sec = make_sections_blockwise(DT, job.count, g, low_bytes, totals.rec_before);
-    // lanes l and l + 16 share a group, so a ballot's two halves OR into the mask of sixteen groups
-    const uint32_t perm = warp * 32 + 2 * (lane & 15) + (lane >> 4);
-    const uint32_t j = 8 * perm;
-    const uint32_t lower = (1u << ((j >> 4) & 31)) - 1;  // groups below this thread's in its mask word
     for (uint32_t k = blockIdx.x; k < g.nblocks; k += gridDim.x) {
         const BlockEntry entry = table[k];
-        const int b = entry.b, n = entry.n, m = entry.m, hbits = n - m;
+        const int b = entry.b, n = entry.n, m = entry.m;
         const bool last = k + 1 == g.nblocks;
         const uint32_t N = last ? g.tail_padded : kBlockElems;
         const uint32_t real = last ? g.tail_real : kBlockElems;
@@ -405,68 +277,10 @@ enec_pack_blocks_kernel(const BlockwiseJob job, int* status) {
         uint8_t* out_smhi = job.out + sec.smhi + uint64_t(k) * (kBlockElems / 8) * 3;
         uint8_t* out_mask = job.out + sec.mask + uint64_t(k) * (kGroupsPerBlock / 8);
         uint8_t* out_rec = job.out + sec.high + entry.rec_before;
-        if (real != kBlockElems) {
+        if (real != kBlockElems)
             pack_tail_block<DT>(in_bytes, N, real, b, n, m, out_sm, out_low, out_smhi, out_mask, out_smlo, out_rec, pack_smem);
-            continue;
-        }
-        const TransformCtx tc = make_transform_ctx(E, b, n);
-        uint2 y[8], hs[8];
-        int bad = 0;
-        uint32_t wide_bits;
-        if (n < 8)
-            wide_bits = encode_full_runs<DT, true>(in_bytes + j * kElemBytes, out_sm + j, out_smlo + j * 2, tc, m, warp, lane, s_mask, y, hs, bad);
         else
-            wide_bits = encode_full_runs<DT, false>(in_bytes + j * kElemBytes, out_sm + j, out_smlo + j * 2, tc, m, warp, lane, s_mask, y, hs, bad);
-        {
-            uint2 ylow[8];
-            const uint32_t lowmask4 = rep4((1u << m) - 1);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) ylow[c] = make_uint2(y[c].x & lowmask4, y[c].y & lowmask4);
-            pack_plane_any(m, smem_u32(s_low), j, N, ylow);
-            if (DT == ENEC_FP16) pack_plane<3>(smem_u32(s_hi3), j, N, hs);
-        }
-        __syncthreads();
-        // wide groups before each mask word and in the block: every warp scans the 32 mask words itself
-        const uint32_t mask_word = s_mask[lane];
-        uint32_t mask_incl = __popc(mask_word);
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, mask_incl, d);
-            if (lane >= uint32_t(d)) mask_incl += t;
-        }
-        const uint32_t mask_excl = mask_incl - __popc(mask_word);
-        const uint32_t wide_count = __shfl_sync(0xFFFFFFFFu, mask_incl, 31);
-        fold_plane_out(smem_u32(s_low), N * uint32_t(m) / 8, out_low, tid);
-        if (DT == ENEC_FP16) fold_plane_out(smem_u32(s_hi3), N * 3 / 8, out_smhi, tid);
-        if (tid < kGroupsPerBlock / 8 / 16) reinterpret_cast<uint4*>(out_mask)[tid] = reinterpret_cast<const uint4*>(s_mask)[tid];
-        if (hbits > 0) {
-            // high bits of wide groups into shared memory, rank order, sixteen value bytes per group; narrow groups
-            // store to a spare slot behind the buffer, so there is no branch
-            const uint32_t hmask4 = rep4(0xFFu >> m);
-            const uint32_t half_off = lane < 16 ? 0 : 8;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t word = ((c * (kBlockElems / 8) + j) >> 9) & 31;
-                const uint32_t rank = __shfl_sync(0xFFFFFFFFu, mask_excl, word) +
-                                      __popc(__shfl_sync(0xFFFFFFFFu, mask_word, word) & lower);
-                sts64(s_exp + (((wide_bits >> c) & 1) ? rank * 16 : kSpare) + half_off,
-                      make_uint2((y[c].x >> m) & hmask4, (y[c].y >> m) & hmask4));
-            }
-            __syncthreads();
-            // Algorithm 2 over each wide group, one group per thread, packed in place: record i lands below the
-            // value bytes of every group that has not been read yet
-            for (uint32_t base = 0; base < wide_count; base += kBlockwiseThreads) {
-                const uint32_t i = base + tid;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (i < wide_count) v = lds128(s_exp + i * 16);
-                __syncthreads();
-                if (i < wide_count) pack_record_any(hbits, v, s_exp + i * 2 * hbits);
-            }
-            __syncthreads();
-            for (uint32_t i = tid; i < wide_count * uint32_t(hbits); i += kBlockwiseThreads)
-                reinterpret_cast<uint16_t*>(out_rec)[i] = uint16_t(lds16(s_exp + 2 * i));
-        }
-        __syncthreads();  // the shared planes and the mask are free for the next block
+            pack_full_block<DT>(in_bytes, b, n, m, out_sm, out_smlo, out_low, out_smhi, out_mask, out_rec, pack_smem, s_mask);
     }
     (void)status;
 }

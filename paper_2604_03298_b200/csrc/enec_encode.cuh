@@ -30,7 +30,7 @@ struct alignas(16) EncodeControl {
     unsigned long long hist[256];  // exponent histogram (2^E bins used)
     uint32_t ticket;               // next block to hand out
     uint32_t hist_done;            // CTAs of the histogram kernel that have finished
-    uint32_t reserved;
+    uint32_t reserved;             // ticket of the kernel that places the records (split form of the compressor)
     int b, n, m;                   // result of the parameter search
     uint8_t lut[256];              // frequency-rank variant: exponent -> rank
     uint8_t unmap[256];            // frequency-rank variant: rank -> exponent (goes into the stream)
@@ -1026,7 +1026,7 @@ enec_encode_kernel(const EncodeJob single, const EncodeBatch batch, int* status)
     if constexpr (!BATCH) {
         if (blockIdx.x == 0) {  // the next call on this scratch area finds its control set zeroed
             single.ctl_next->hist[tid] = 0;
-            if (tid == 0) { single.ctl_next->ticket = 0; single.ctl_next->hist_done = 0; }
+            if (tid == 0) { single.ctl_next->ticket = 0; single.ctl_next->hist_done = 0; single.ctl_next->reserved = 0; }
         }
         fill_tensor_ctx<DT, RANKED>(single, single_tensor, single_tc);
         if constexpr (RANKED) {  // the exponent -> rank table of the tensor, for every block of this CTA
