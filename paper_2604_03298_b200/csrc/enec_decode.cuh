@@ -242,12 +242,14 @@ __device__ inline int load_job(const DecodeJob& job, JobCtx& c, bool blockwise =
 // expanded records: sixteen bytes per wide group (its high bits, one element per byte), rank order, and
 // one more slot at index cap that the rank entries of narrow groups point to in blocks that fit.
 // cap = records per block that fit; records beyond it are read from global memory by the consumers.
+// nibble: the expanded records take eight bytes each (n - m <= 4: byte j of a record's two words holds element j in
+// its low and element j + 4 in its high half), which lets full blocks with many wide groups still fit.
 struct StageLayout {
     uint32_t mask, rank, low, smhi, sm, raw, expanded, cap, bytes;
 };
 constexpr uint32_t kStageRankTable = kStageBytes - kRankTableBytes;  // where a stage keeps a stream's rank table
 // mapped: the stage also holds the stream's rank -> exponent table (its last 256 bytes).
-__host__ __device__ inline StageLayout make_stage_layout(int dt, int m, int hbits, bool mapped = false) {
+__host__ __device__ inline StageLayout make_stage_layout(int dt, int m, int hbits, bool mapped = false, bool nibble = false) {
     StageLayout L;
     const uint32_t usable = mapped ? kStageRankTable : kStageBytes;
     L.mask = kStageMetaBytes;
@@ -256,11 +258,12 @@ __host__ __device__ inline StageLayout make_stage_layout(int dt, int m, int hbit
     L.smhi = L.low + kBlockElems * uint32_t(m) / 8;
     L.sm = L.smhi + (dt == ENEC_FP16 ? kBlockElems * 3 / 8 : 0);
     L.raw = L.sm + kBlockElems;  // at most 35072 (m = 8, or fp16 with m = 5), so a stage always has room
-    uint32_t cap = hbits > 0 ? (usable - L.raw - 64) / uint32_t(2 * hbits + 16) : 0;
+    const uint32_t expanded_size = nibble ? 8 : 16;
+    uint32_t cap = hbits > 0 ? (usable - L.raw - 64) / (uint32_t(2 * hbits) + expanded_size) : 0;
     if (cap > kGroupsPerBlock) cap = kGroupsPerBlock;
     L.cap = cap;
     L.expanded = L.raw + uint32_t(align16(uint64_t(cap) * 2 * hbits + 32));
-    L.bytes = L.expanded + (cap + 1) * 16;
+    L.bytes = L.expanded + (cap + 1) * expanded_size;
     return L;
 }
 static_assert(kStageMetaBytes + kGroupsPerBlock / 8 + kGroupsPerBlock * 2 + 2 * kBlockElems + 64 + kRankTableBytes <= kStageBytes,
@@ -279,6 +282,19 @@ struct RunCtx {
     uint32_t c4;                    // rep4(b + 2^(n-1)) when that sum fits a byte
     int n;
 };
+
+// The eight-byte form of the expanded records exists in the fp16 kernel only: fp16 weights have five exponent
+// bits and (n, m) = (5, 3), so half of their groups can be wide, more than a stage holds in the sixteen-byte form;
+// the bf16 and fp32 kernels, whose blocks fit, carry none of its code (measured: with it their one-stream rate
+// fell by 1.5 to 4 %, from code layout alone).
+template <int DT, bool MAPPED>
+constexpr bool kNibbleForm = DT == ENEC_FP16 && !MAPPED;
+
+// Whether x = (b + 2^(n-1)) - (y ^ 2^(n-1)) can be taken as one subtraction per word (what the branch-free bodies do).
+template <int DT>
+__host__ __device__ inline bool plain_subtraction(uint32_t b, uint32_t n) {
+    return DT == ENEC_FP16 || n == 8 || b + (1u << (n - 1)) <= 255;
+}
 
 // Inverse transform on four packed bytes: x = (b - sext_n(y)) mod 2^E  (Sec. 5.3).
 // sext_n(y) = (y ^ s) - s with s = 2^(n-1), so x = (b + s) - (y ^ s) per byte.
@@ -432,12 +448,13 @@ __device__ __forceinline__ void decode_block(const RunCtx& r, uint32_t s_low, ui
 // The frequency-rank variant (MAPPED) has no sign position: nothing is flipped, the slot of narrow groups holds
 // zeros, and the exponent comes from the stage's rank table (shared address in r.c4) instead of the subtraction.
 // tid = 0..255; thread tid owns the runs c * 2048 + 8 tid (c < 8).
-template <int DT, int M, int HB, bool MAPPED = false>
+// NIBBLE: the expanded records are in the eight-byte form (see StageLayout).
+template <int DT, int M, int HB, bool MAPPED = false, bool NIBBLE = false>
 __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_low, uint32_t s_smhi, uint32_t tid) {
     constexpr int n = M + HB;
     constexpr uint32_t Hm = 0x80808080u;
     const uint32_t rank_addr = r.rank + (tid >> 1) * 2;
-    const uint32_t exp_addr = r.expanded + (tid & 1) * 8;
+    const uint32_t exp_addr = r.expanded + (tid & 1) * (NIBBLE ? 4 : 8);
     const uint32_t sm_addr = r.sm + 8 * tid;
     uint4* out = reinterpret_cast<uint4*>(r.out + 8 * tid);
     [[maybe_unused]] uint32_t* out32 = reinterpret_cast<uint32_t*>(r.out) + 8 * tid;
@@ -465,7 +482,14 @@ __device__ __forceinline__ void decode_full_block(const RunCtx& r, uint32_t s_lo
         }
         if constexpr (HB > 0) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) hi[q] = lds64(exp_addr + rk[4 * h + q] * 16);
+            for (int q = 0; q < 4; ++q) {
+                if constexpr (NIBBLE) {
+                    const uint32_t w = lds32(exp_addr + rk[4 * h + q] * 8);
+                    hi[q] = make_uint2(w & 0x0F0F0F0Fu, (w >> 4) & 0x0F0F0F0Fu);
+                } else {
+                    hi[q] = lds64(exp_addr + rk[4 * h + q] * 16);
+                }
+            }
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) smv[q] = lds64(sm_addr + (4 * h + q) * (kBlockElems / 8));
@@ -555,25 +579,28 @@ __device__ __forceinline__ uint32_t build_rank_array(uint32_t s_mask, uint32_t s
 
 // The staged records expanded to sixteen bytes each (one value per byte), all consumer threads.
 // `flip` is XORed into every expanded word (the branch-free body wants the sign position flipped).
+// nibble: eight bytes per record instead (values below 16: elements 0..3 and 8..11 in the low halves of the two words'
+// bytes, elements 4..7 and 12..15 in the high halves).
 template <int HB>
 __device__ __forceinline__ void expand_records(uint32_t s_raw, uint32_t s_expanded, uint32_t count, uint32_t tid,
-                                               uint32_t flip) {
+                                               uint32_t flip, bool nibble = false) {
     for (uint32_t i = tid; i < count; i += kConsumerWarps * 32) {
         const uint32_t rp = s_raw + i * (2 * HB);
         uint4 v = unpack_record<HB>([&](int w) { return lds16(rp + 2 * w); });
         v.x ^= flip; v.y ^= flip; v.z ^= flip; v.w ^= flip;
-        sts128(s_expanded + i * 16, v);
+        if (HB <= 4 && nibble) sts64(s_expanded + i * 8, make_uint2(v.x | (v.y << 4), v.z | (v.w << 4)));
+        else sts128(s_expanded + i * 16, v);
     }
 }
 
 __device__ __forceinline__ void expand_records_any(int hbits, uint32_t s_raw, uint32_t s_expanded, uint32_t count,
-                                                   uint32_t tid, uint32_t flip) {
+                                                   uint32_t tid, uint32_t flip, bool nibble = false) {
     switch (hbits) {
         case 0: break;
-        case 1: expand_records<1>(s_raw, s_expanded, count, tid, flip); break;
-        case 2: expand_records<2>(s_raw, s_expanded, count, tid, flip); break;
-        case 3: expand_records<3>(s_raw, s_expanded, count, tid, flip); break;
-        case 4: expand_records<4>(s_raw, s_expanded, count, tid, flip); break;
+        case 1: expand_records<1>(s_raw, s_expanded, count, tid, flip, nibble); break;
+        case 2: expand_records<2>(s_raw, s_expanded, count, tid, flip, nibble); break;
+        case 3: expand_records<3>(s_raw, s_expanded, count, tid, flip, nibble); break;
+        case 4: expand_records<4>(s_raw, s_expanded, count, tid, flip, nibble); break;
         case 5: expand_records<5>(s_raw, s_expanded, count, tid, flip); break;
         case 6: expand_records<6>(s_raw, s_expanded, count, tid, flip); break;
         default: expand_records<7>(s_raw, s_expanded, count, tid, flip); break;
@@ -626,7 +653,7 @@ struct BlockDesc {
     uint32_t expect;    // wide groups of the block according to the prefix table
     uint32_t N;         // padded block length
     uint32_t real;      // real elements
-    uint32_t code;      // m * 8 + (n - m); bit 8: frequency-rank variant (the stage then holds the rank table)
+    uint32_t code;      // m * 8 + (n - m); bit 7: the expanded records take the eight-byte form
     uint32_t b, n;
     StageLayout L;
     uint16_t* out;        // global: first element of the block
@@ -854,8 +881,17 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
                 failed = true;
                 break;
             }
+            // a full block with more wide groups than the stage holds in the sixteen-byte form takes the eight-byte
+            // form when that holds them all (and its consumers will take the branch-free body)
+            StageLayout Lb = L;
+            bool nibble = false;
+            if (kNibbleForm<DT, MAPPED> && hbits >= 1 && hbits <= 4 && expect > L.cap && real == kBlockElems &&
+                plain_subtraction<DT>(uint32_t(blk_b), uint32_t(blk_n))) {
+                const StageLayout L8 = make_stage_layout(DT, blk_m, hbits, false, true);
+                if (expect <= L8.cap) { Lb = L8; nibble = true; }
+            }
             const uint64_t w0 = h0 & ~uint64_t(15);
-            uint32_t staged = expect < L.cap ? expect : L.cap;  // records staged in shared memory
+            uint32_t staged = expect < Lb.cap ? expect : Lb.cap;  // records staged in shared memory
             if (hbits == 0) staged = 0;
             const uint64_t w1 = align16(h0 + uint64_t(staged) * (2 * hbits));
             const uint32_t mask_bytes = uint32_t(align16(((N >> 4) + 7) / 8));
@@ -870,10 +906,10 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             d->expect = expect;
             d->N = N;
             d->real = real;
-            d->code = uint32_t(blk_m * 8 + hbits);
+            d->code = uint32_t(blk_m * 8 + hbits) | (nibble ? 128u : 0u);
             d->b = uint32_t(blk_b);
             d->n = uint32_t(blk_n);
-            d->L = L;
+            d->L = Lb;
             d->out = jc.out + uint64_t(k) * kBlockElems * (DT == ENEC_FP32 ? 2 : 1);
             if (DT == ENEC_FP32) {
                 // the low halves go from global memory straight to the consumers' registers: start them
@@ -888,12 +924,12 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             mbar_expect_tx(&ctl->full[s], mask_bytes + low_bytes + smhi_bytes + sm_bytes + raw_bytes +
                                               (MAPPED ? kRankTableBytes : 0u));
             if constexpr (MAPPED) bulk_g2s(st + kStageRankTable, jc.in + kHeaderBytes, kRankTableBytes, &ctl->full[s]);
-            bulk_g2s(st + L.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
-            bulk_g2s(st + L.low, jc.in + low_src, low_bytes, &ctl->full[s]);
+            bulk_g2s(st + Lb.mask, jc.in + jc.off_mask + uint64_t(k) * (kGroupsPerBlock / 8), mask_bytes, &ctl->full[s]);
+            bulk_g2s(st + Lb.low, jc.in + low_src, low_bytes, &ctl->full[s]);
             if (DT == ENEC_FP16)
-                bulk_g2s(st + L.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
-            bulk_g2s(st + L.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
-            if (raw_bytes) bulk_g2s(st + L.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
+                bulk_g2s(st + Lb.smhi, jc.in + jc.off_smhi + uint64_t(k) * (kBlockElems / 8) * 3, smhi_bytes, &ctl->full[s]);
+            bulk_g2s(st + Lb.sm, jc.in + jc.off_sm + uint64_t(k) * kBlockElems, sm_bytes, &ctl->full[s]);
+            if (raw_bytes) bulk_g2s(st + Lb.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
             if (!jc.blockwise && k + 2 <= jc.nblocks) t2 = table[k + 2];  // for the tensor's next block
         }
         if (failed) {
@@ -919,26 +955,30 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             break;
         }
         const BlockDesc* d = reinterpret_cast<const BlockDesc*>(smem + sizeof(DecodeShared) + size_t(s) * kStageBytes);
-        const uint32_t N = d->N, expect = d->expect, code = d->code;
+        const uint32_t N = d->N, expect = d->expect, code = kNibbleForm<DT, MAPPED> ? d->code & 127u : d->code;
+        const bool nibble = kNibbleForm<DT, MAPPED> && (d->code & 128u) != 0;  // only set for blocks that take the branch-free body
         const uint32_t b = d->b, n = d->n;
         const uint32_t hbits = code & 7;
         const uint32_t cap = d->L.cap;
         const uint32_t o_rank = d->L.rank, o_low = d->L.low, o_smhi = d->L.smhi, o_sm = d->L.sm, o_raw = d->L.raw,
                        o_exp = d->L.expanded;
         const uint32_t sbit = 1u << (n - 1);
-        const bool simple_sub = DT == ENEC_FP16 || n == 8 || b + sbit <= 255;
+        const bool simple_sub = plain_subtraction<DT>(b, n);
         const bool full_block = N == kBlockElems && d->real == kBlockElems && expect <= cap && (MAPPED || simple_sub);
         // preparation: ranks of the wide groups and expanded records
         if (hbits > 0) {
             // the branch-free body wants narrow groups to point at the flip slot and flipped records
             const uint32_t flip4 = MAPPED ? 0u : rep4(1u << (hbits - 1));
-            if (tid == 0) sts128(st + o_exp + cap * 16, make_uint4(flip4, flip4, flip4, flip4));
+            if (tid == 0) {
+                if (nibble) sts64(st + o_exp + cap * 8, make_uint2(flip4 | (flip4 << 4), flip4 | (flip4 << 4)));
+                else sts128(st + o_exp + cap * 16, make_uint4(flip4, flip4, flip4, flip4));
+            }
             const uint32_t wide = build_rank_array(st + d->L.mask, st + o_rank, N, tid, full_block ? cap : kNotWide);
             if (wide != expect && lane == 0) {  // the prefix table must agree with the mask
                 *abort_flag = 1;
                 report(status, ENEC_ERR_BAD_STREAM);
             }
-            expand_records_any(int(hbits), st + o_raw + d->first, st + o_exp, d->staged, tid, full_block ? flip4 : 0);
+            expand_records_any(int(hbits), st + o_raw + d->first, st + o_exp, d->staged, tid, full_block ? flip4 : 0, nibble);
         }
         RunCtx r;
         {
@@ -960,6 +1000,21 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             r.real = d->real;
         }
         if (consumer_barrier_or(*abort_flag != 0)) break;
+        if (nibble) {  // a full block with more wide groups than the sixteen-byte form holds
+            if constexpr (kNibbleForm<DT, MAPPED>) {
+                switch (code) {
+#define ENEC_CASE(DTV, MV, HV)                                                               \
+    case MV * 8 + HV:                                                                        \
+        if constexpr (HV >= 1 && HV <= 4 && (DTV != ENEC_FP16 || MV + HV <= 5))               \
+            decode_full_block<DTV, MV, HV, false, true>(r, st + o_low, st + o_smhi, tid);    \
+        break;
+                    ENEC_FOR_EACH_MH(ENEC_CASE, DT)
+                    ENEC_FOR_EACH_MH_BF16_ONLY(ENEC_CASE, DT)
+#undef ENEC_CASE
+                    default: break;
+                }
+            }
+        } else
         switch (code) {
 #define ENEC_CASE(DTV, MV, HV)                                                               \
     case MV * 8 + HV:                                                                        \
