@@ -136,26 +136,20 @@ __host__ __device__ inline int width_eq1(int b, int l, int h, int E) {
     return n;
 }
 
-// Eq. 4 at L = 16 for every m in 1..n, given the number of elements per bit width of the stored value; one
-// thread. Plain IEEE double, one rounding per operation, no fused multiply-add; ties go to the smaller m.
-__device__ __forceinline__ int choose_m(const unsigned long long (&width_count)[9], int n) {
+// Eq. 4 at L = 16 for one m in 1..n, given the number of elements per bit width of the stored value. Plain IEEE
+// double, one rounding per operation, no fused multiply-add.
+__device__ __forceinline__ double expected_bits(const unsigned long long* width_count, int n, int m) {
     unsigned long long total = 0;
     for (int w = 0; w <= 8; ++w) total += width_count[w];
-    unsigned long long cnt = width_count[0];
-    int best_m = 1;
-    double best_bits = 0.0;
-    for (int m = 1; m <= n; ++m) {
-        cnt += width_count[m];
-        const double p = __ddiv_rn(__ull2double_rn(cnt), __ull2double_rn(total));
-        const double p2 = __dmul_rn(p, p);
-        const double p4 = __dmul_rn(p2, p2);
-        const double p8 = __dmul_rn(p4, p4);
-        const double p16 = __dmul_rn(p8, p8);
-        const double saving = __dmul_rn(double(m - n), p16);
-        const double bits = __dadd_rn(__dadd_rn(double(n), 0.0625), saving);  // 1/L + n + (m - n) p^L
-        if (m == 1 || bits < best_bits) { best_m = m; best_bits = bits; }
-    }
-    return best_m;
+    unsigned long long cnt = 0;
+    for (int w = 0; w <= m; ++w) cnt += width_count[w];
+    const double p = __ddiv_rn(__ull2double_rn(cnt), __ull2double_rn(total));
+    const double p2 = __dmul_rn(p, p);
+    const double p4 = __dmul_rn(p2, p2);
+    const double p8 = __dmul_rn(p4, p4);
+    const double p16 = __dmul_rn(p8, p8);
+    const double saving = __dmul_rn(double(m - n), p16);
+    return __dadd_rn(__dadd_rn(double(n), 0.0625), saving);  // 1/L + n + (m - n) p^L
 }
 
 // Sec. 5.5 phases 2 and 3 on a finished histogram; threads 0..255 of one CTA, thread t bringing the count of
@@ -168,6 +162,7 @@ __device__ void parameter_search_counts(unsigned long long mine, int& out_b, int
     __shared__ unsigned long long s_hist[256];
     __shared__ unsigned long long s_key[kHistThreads / 32];
     __shared__ unsigned long long s_width_count[9];
+    __shared__ double s_bits[8];
     __shared__ int s_lo, s_hi, s_b, s_n, s_m;
     const uint32_t tid = threadIdx.x;
     s_hist[tid] = tid < uint32_t(kBins) ? mine : 0ull;
@@ -208,7 +203,16 @@ __device__ void parameter_search_counts(unsigned long long mine, int& out_b, int
         atomicAdd(&s_width_count[bit_width_u32(y)], s_hist[tid]);
     }
     __syncthreads();
-    if (tid == 0) s_m = choose_m(s_width_count, n);
+    // Eq. 4: thread m - 1 evaluates m (the double-precision chain is long, so the candidates run side by side);
+    // thread 0 takes the smallest value, the smaller m on ties
+    if (tid < uint32_t(n)) s_bits[tid] = expected_bits(s_width_count, n, int(tid) + 1);
+    __syncthreads();
+    if (tid == 0) {
+        int best_m = 1;
+        for (int m = 2; m <= n; ++m)
+            if (s_bits[m - 1] < s_bits[best_m - 1]) best_m = m;
+        s_m = best_m;
+    }
     __syncthreads();
     out_b = b;
     out_n = n;
@@ -260,7 +264,13 @@ __device__ void parameter_search_ranked(EncodeControl* ctl) {
         const int n = s_occupied <= 1 ? 1 : bit_width_u32(s_occupied - 1);
         ctl->b = 0;
         ctl->n = n;
-        ctl->m = choose_m(s_width_count, n);
+        int best_m = 1;
+        double best_bits = expected_bits(s_width_count, n, 1);
+        for (int m = 2; m <= n; ++m) {  // ties go to the smaller m
+            const double bits = expected_bits(s_width_count, n, m);
+            if (bits < best_bits) { best_m = m; best_bits = bits; }
+        }
+        ctl->m = best_m;
     }
 }
 

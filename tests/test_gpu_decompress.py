@@ -157,3 +157,27 @@ def test_fp16_full_width_field(oracle):
                  | (rng.integers(0, 2, count).astype(np.uint16) << 15)).astype(np.uint16)
         for m in (1, 3, 5):
             check_roundtrip(oracle, words, 1, (b, 5, m))
+
+
+@pytest.mark.parametrize("n,m", [(5, 3), (5, 1), (4, 2), (5, 4), (3, 1)])
+def test_fp16_blocks_with_many_wide_groups(oracle, n, m):
+    """fp16 blocks whose number of wide groups runs from below what a stage holds as sixteen-byte records, through the
+    range of the eight-byte form, up to every group: one block per count, with exact per-block counts."""
+    rng = np.random.default_rng(10 * n + m)
+    b = 12
+    wide_counts = [0, 1, 300, 392, 393, 394, 500, 610, 640, 655, 656, 657, 700, 900, 1023, 1024]
+    blocks = []
+    for wide in wide_counts:
+        # narrow values keep y = b - x below 2^m; one element of each chosen group gets a y with a high bit set
+        y = rng.integers(0, 1 << m, 16384)
+        groups = rng.choice(1024, size=wide, replace=False)
+        spots = groups * 16 + rng.integers(0, 16, wide)
+        y[spots] = rng.integers(1 << m, 1 << (n - 1), wide) if n - 1 > m else (1 << m)
+        x = (b - y) & 31
+        blocks.append(((x.astype(np.uint16) << 10) | rng.integers(0, 1024, 16384).astype(np.uint16)
+                       | (rng.integers(0, 2, 16384).astype(np.uint16) << 15)).astype(np.uint16))
+    words = np.concatenate(blocks + [blocks[3][:5000]])
+    stream = oracle.compress(words, 1, (b, n, m))
+    table = np.frombuffer(stream[64:64 + 4 * (len(wide_counts) + 2)].tobytes(), dtype=np.uint32)
+    assert np.diff(table)[:len(wide_counts)].tolist() == wide_counts
+    check_roundtrip(oracle, words, 1, (b, n, m))
