@@ -1,6 +1,6 @@
 """Seeded random cases, GPU against the oracle: random dtype, size (0 .. 600 K values, around block boundaries),
 value distribution (Gaussian at random scales, Student-t, shifted, with zeros, constant, random bit patterns) and
-entry point (single, allocation-free, batched). Streams byte for byte, decoded tensors bit for bit."""
+entry point (single, allocation-free, batched, frequency-rank, block-wise). Streams byte for byte, decoded tensors bit for bit."""
 import numpy as np
 import pytest
 import torch
@@ -116,6 +116,38 @@ def test_ranked_calls(oracle, seed):
         out = torch.empty(count + 16, dtype=TD[dt], device="cuda")
         d_want = torch.from_numpy(want).cuda()
         assert enec.enec_decompress_ranked(d_want, d_want.numel(), dt, count, out, status) == 0
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, (seed, case, dt, count)
+        got = buf[:int(size.item())].cpu().numpy()
+        assert got.size == want.size and np.array_equal(got, want), (seed, case, dt, count)
+        assert (buf[cap:] == 0xA5).all()
+        assert np.array_equal(from_dev(out[:count], dt, w), w), (seed, case, dt, count)
+
+
+@pytest.mark.parametrize("seed", [41, 42])
+def test_blockwise_calls(oracle, seed):
+    """The variant with parameters per block over the same random inputs; every second tensor is cut into stretches
+    of different scale, so that the blocks' searches disagree."""
+    import paper_2604_03298_b200 as enec
+    rng = np.random.default_rng(seed)
+    for case in range(80):
+        dt = int(rng.integers(0, 3))
+        count = max(0, int(rng.choice([rng.integers(0, 200), rng.integers(0, 40000), rng.integers(0, 400000),
+                                       16384 * int(rng.integers(1, 20)) + int(rng.integers(-2, 3))])))
+        w = draw(rng, dt, count)
+        if case % 2 and count > 40000:
+            other = draw(rng, dt, count)
+            cut = int(rng.integers(1, count))
+            w = np.concatenate([w[:cut], other[cut:]])
+        want = oracle.compress_blockwise(w, dt)
+        cap = enec.enec_max_compressed_size_blockwise(dt, count)
+        buf = torch.full((cap + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+        size = torch.zeros(1, dtype=torch.int64, device="cuda")
+        status = status_tensor()
+        assert enec.enec_compress_blockwise(to_dev(w, dt), dt, count, buf, cap, size, status) == 0
+        out = torch.empty(count + 16, dtype=TD[dt], device="cuda")
+        d_want = torch.from_numpy(want).cuda()
+        assert enec.enec_decompress_blockwise(d_want, d_want.numel(), dt, count, out, status) == 0
         torch.cuda.synchronize()
         assert int(status.item()) == 0, (seed, case, dt, count)
         got = buf[:int(size.item())].cpu().numpy()
