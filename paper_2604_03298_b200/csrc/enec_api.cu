@@ -450,9 +450,9 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
     if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
     if (n_items < 0 || (n_items > 0 && !h_items)) return ENEC_ERR_INVALID_ARG;
     if (n_items == 0) return ENEC_OK;
-    // descriptors and block prefix in one host buffer: [jobs | prefix]
+    // descriptors and block prefix in one host buffer: [jobs | prefix]; long lists add [ticket | tensor of every chunk]
     const size_t jobs_bytes = size_t(n_items) * sizeof(DecodeJob);
-    const size_t prefix_bytes = (size_t(n_items) + 1) * sizeof(uint32_t);
+    const size_t prefix_bytes = size_t(ticket_offset_behind_prefix(uint32_t(n_items)));
     std::vector<uint8_t> host(jobs_bytes + prefix_bytes);
     DecodeJob* jobs = reinterpret_cast<DecodeJob*>(host.data());
     uint32_t* prefix = reinterpret_cast<uint32_t*>(host.data() + jobs_bytes);
@@ -494,6 +494,7 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
     batch.n_jobs = uint32_t(n_items);
     batch.blockwise = 0;
     batch.total_blocks = uint32_t(total);
+    bool ticketed = false;
     if (uint32_t(n_items) <= kInlineJobs) {
         // a short list travels in the launch parameters: no copy, no scratch
         batch.jobs = nullptr;
@@ -501,6 +502,21 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
         for (int i = 0; i < n_items; ++i) batch.inline_jobs[i] = jobs[i];
         for (int i = 0; i <= n_items; ++i) batch.inline_prefix[i] = prefix[i];
     } else {
+        // the blocks of a long list are handed out in chunks: a zeroed ticket word and the tensor of every chunk's
+        // first block travel with the descriptors
+        const size_t ticket_at = host.size();
+        const size_t n_chunks = size_t((total + kTicketChunk - 1) / kTicketChunk);
+        host.resize(ticket_at + 16 + n_chunks * sizeof(uint32_t), 0);
+        {
+            const uint32_t* pre = reinterpret_cast<const uint32_t*>(host.data() + jobs_bytes);
+            uint32_t* chunk_job = reinterpret_cast<uint32_t*>(host.data() + ticket_at + 16);
+            uint32_t j = 0;
+            for (size_t c = 0; c < n_chunks; ++c) {
+                const uint64_t first = uint64_t(c) * kTicketChunk;
+                while (pre[j + 1] <= first) ++j;  // tensors without blocks are skipped
+                chunk_job[c] = j;
+            }
+        }
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
         uint8_t* scratch = nullptr;
@@ -511,8 +527,9 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
             return ENEC_ERR_CUDA;
         batch.jobs = reinterpret_cast<const DecodeJob*>(scratch);
         batch.prefix = reinterpret_cast<const uint32_t*>(scratch + jobs_bytes);
+        ticketed = n_chunks > 0;
     }
-    return launch_decode_any(dt, batch, d_status, stream, false);
+    return launch_decode_any(dt, batch, d_status, stream, false, ticketed);
 }
 
 enec_status enec_compress(const void* d_in, enec_dtype dt, size_t count, void* d_out, size_t out_capacity,

@@ -665,7 +665,15 @@ static_assert(sizeof(BlockDesc) <= kStageMetaBytes, "descriptor fits the stage's
 constexpr uint32_t kInlineJobs = 16;  // tensors of a short batch that fit the kernel's parameter space
 
 // A launch decodes the blocks of one tensor or of a list of tensors. Blocks of all tensors form one
-// index space; a CTA takes a contiguous range of it, so it changes tensor rarely.
+// index space; a CTA takes a contiguous range of it, so it changes tensor rarely. Long lists (the kernel instance
+// with TICKET) hand the index space out in chunks of kTicketChunk consecutive blocks instead: the CTAs of an SM
+// progress unequally, and with a fixed share each the launch ends when the slowest has finished. Such a list's
+// device arrays are laid out as [jobs | prefix, padded to 16 bytes | ticket word, 16 bytes, zero at launch | the
+// tensor of every chunk's first block], so the kernel finds the last two behind the prefix.
+constexpr uint32_t kTicketChunk = 8;
+__host__ __device__ inline uint64_t ticket_offset_behind_prefix(uint32_t n_jobs) {
+    return align16((uint64_t(n_jobs) + 1) * sizeof(uint32_t));
+}
 struct DecodeBatch {
     const DecodeJob* jobs;    // device array, or null when the tensors travel inside the launch parameters
     const uint32_t* prefix;   // device array [n_jobs + 1]: blocks before each tensor (null with jobs)
@@ -733,8 +741,9 @@ __device__ __forceinline__ void prefetch_before_wait(const DecodeBatch& batch, u
 }
 
 // MAPPED: the instance for streams of the frequency-rank variant (general block body with table look-ups only);
-// each instance refuses the other kind of stream.
-template <int DT, bool MAPPED = false>
+// each instance refuses the other kind of stream. TICKET: blocks are handed out by batch.ticket; the loader ends the
+// consumers' loop with a descriptor of zero length.
+template <int DT, bool MAPPED = false, bool TICKET = false>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
 enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -782,7 +791,28 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
         uint32_t j = 0;
         const DecodeJob* jobs = batch.jobs ? batch.jobs : batch.inline_jobs;
         const uint32_t* prefix = batch.jobs ? batch.prefix : batch.inline_prefix;
-        {
+        // TICKET: the chunk in hand, the one after it (asked for a chunk ahead, so that the answer is there in time),
+        // and the blocks of the chunk in hand that are issued
+        [[maybe_unused]] uint32_t chunk = 0, next_chunk = 0, in_chunk = 0;
+        [[maybe_unused]] uint32_t next_j = 0, next_first = 0, next_end = 0;  // the next chunk's tensor and its range of blocks
+        [[maybe_unused]] const uint32_t n_chunks = TICKET ? (batch.total_blocks + kTicketChunk - 1) / kTicketChunk : 0;
+        [[maybe_unused]] uint32_t* const ticket =
+            TICKET ? reinterpret_cast<uint32_t*>(reinterpret_cast<uintptr_t>(batch.prefix) + ticket_offset_behind_prefix(batch.n_jobs))
+                   : nullptr;
+        [[maybe_unused]] const uint32_t* const chunk_job = TICKET ? ticket + 4 : nullptr;
+        [[maybe_unused]] auto look_up_next = [&]() {
+            if (next_chunk < n_chunks) {
+                next_j = chunk_job[next_chunk];
+                next_first = prefix[next_j];
+                next_end = prefix[next_j + 1];
+            }
+        };
+        if constexpr (TICKET) {
+            chunk = atomicAdd(ticket, 1u);
+            next_chunk = atomicAdd(ticket, 1u);
+            if (chunk < n_chunks) j = chunk_job[chunk];
+            look_up_next();
+        } else {
             uint32_t lo = 0, hi = batch.n_jobs;  // largest j with prefix[j] <= first_block
             while (hi - lo > 1) {
                 const uint32_t mid = (lo + hi) >> 1;
@@ -800,8 +830,26 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
         uint32_t t1 = 0, t2 = 0;  // table[k + 1], table[k + 2] of the block about to be issued (one ahead)
         uint32_t issued = 0;
         bool failed = false;
-        for (; issued < n_mine; ++issued) {
-            const uint32_t gb = first_block + issued;
+        for (; TICKET || issued < n_mine; ++issued) {
+            uint32_t gb = first_block + issued;
+            [[maybe_unused]] bool jumped = false;  // TICKET: this block does not follow the one issued before it
+            if constexpr (TICKET) {
+                if (in_chunk == kTicketChunk) {
+                    chunk = next_chunk;
+                    if (chunk >= n_chunks) break;
+                    if (next_j != j) parsed = false;
+                    j = next_j;
+                    job_first = next_first;
+                    job_end = next_end;
+                    next_chunk = atomicAdd(ticket, 1u);
+                    look_up_next();
+                    in_chunk = 0;
+                    jumped = true;
+                }
+                gb = chunk * kTicketChunk + in_chunk;
+                ++in_chunk;
+                if (chunk >= n_chunks || gb >= batch.total_blocks) break;
+            }
             while (gb >= job_end) {  // next tensor (tensors without blocks are skipped)
                 ++j;
                 job_first = job_end;
@@ -841,6 +889,12 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             } else {
                 t0 = t1;
                 t1 = t2;
+                if constexpr (TICKET) {
+                    if (jumped) {
+                        t0 = table[k];
+                        t1 = table[k + 1];
+                    }
+                }
             }
             const uint32_t s = issued % S, use = issued / S;
             if (use > 0 && !suspended_wait(&ctl->empty[s], (use - 1) & 1, abort_flag)) { failed = true; break; }
@@ -932,6 +986,18 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             if (raw_bytes) bulk_g2s(st + Lb.raw, jc.in + w0, raw_bytes, &ctl->full[s]);
             if (!jc.blockwise && k + 2 <= jc.nblocks) t2 = table[k + 2];  // for the tensor's next block
         }
+        if constexpr (TICKET) {
+            if (!failed) {  // tell the consumers that this was the last block
+                const uint32_t s = issued % S, use = issued / S;
+                if (use > 0 && !suspended_wait(&ctl->empty[s], (use - 1) & 1, abort_flag)) {
+                    failed = true;
+                } else {
+                    BlockDesc* d = reinterpret_cast<BlockDesc*>(smem + sizeof(DecodeShared) + size_t(s) * kStageBytes);
+                    d->N = 0;
+                    mbar_expect_tx(&ctl->full[s], 0u);
+                }
+            }
+        }
         if (failed) {
             if (!*abort_flag) { *abort_flag = 1; report(status, ENEC_ERR_TIMEOUT); }
             // let copies still in flight land before the CTA's shared memory is released
@@ -943,7 +1009,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
 
     // ---------------- consumers ----------------
     const uint32_t tid = threadIdx.x;
-    for (uint32_t i = 0; i < n_mine; ++i) {
+    for (uint32_t i = 0; TICKET || i < n_mine; ++i) {
         const uint32_t s = i % S, use = i / S;
         const uint32_t st = stages + s * kStageBytes;
         // every consumer thread waits on the stage's mbarrier itself; the wait suspends the thread in hardware,
@@ -955,6 +1021,7 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             break;
         }
         const BlockDesc* d = reinterpret_cast<const BlockDesc*>(smem + sizeof(DecodeShared) + size_t(s) * kStageBytes);
+        if (TICKET && d->N == 0) break;  // the loader's end mark
         const uint32_t N = d->N, expect = d->expect, code = kNibbleForm<DT, MAPPED> ? d->code & 127u : d->code;
         const bool nibble = kNibbleForm<DT, MAPPED> && (d->code & 128u) != 0;  // only set for blocks that take the branch-free body
         const uint32_t b = d->b, n = d->n;

@@ -24,7 +24,8 @@ inline DecodeDevice* decode_device(int dev) {
 }
 
 template <int DT>
-inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked = false) {
+inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked = false,
+                                 bool ticketed = false) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
     DecodeDevice* found = decode_device(dev);
@@ -34,6 +35,8 @@ inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaSt
         if (cudaFuncSetAttribute(enec_decode_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(kDecodeSmemBytes)) != cudaSuccess ||
             cudaFuncSetAttribute(enec_decode_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(kDecodeSmemBytes)) != cudaSuccess ||
+            cudaFuncSetAttribute(enec_decode_kernel<DT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(kDecodeSmemBytes)) != cudaSuccess)
             return ENEC_ERR_CUDA;
         info.attr_set[DT] = true;
@@ -42,15 +45,17 @@ inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaSt
     if (grid > batch.total_blocks) grid = batch.total_blocks;
     if (grid == 0) grid = 1;
     const cudaError_t err =
-        ranked ? launch_pdl(enec_decode_kernel<DT, true>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status)
-               : launch_pdl(enec_decode_kernel<DT, false>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status);
+        ranked         ? launch_pdl(enec_decode_kernel<DT, true>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status)
+        : ticketed     ? launch_pdl(enec_decode_kernel<DT, false, true>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch,
+                                    d_status)
+                       : launch_pdl(enec_decode_kernel<DT, false>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
 
 
-enec_status launch_decode_bf16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked);
-enec_status launch_decode_fp16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked);
-enec_status launch_decode_fp32(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked);
+enec_status launch_decode_bf16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, bool ticketed);
+enec_status launch_decode_fp16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, bool ticketed);
+enec_status launch_decode_fp32(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, bool ticketed);
 
 }  // namespace enec

@@ -14,7 +14,9 @@ constexpr int kMaxDevices = 64;  // device ordinals the per-device tables cover;
 
 struct DecodeBatch;
 // Launches the decode kernel instance for dt (and for the frequency-rank variant when ranked) over `batch`.
-enec_status launch_decode_any(int dt, const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked);
+// ticketed: the batch's device arrays carry a ticket word and the chunk table (see DecodeBatch).
+enec_status launch_decode_any(int dt, const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked,
+                              bool ticketed = false);
 
 // Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
 // stream drains; it waits for the predecessor's completion itself (pdl_wait) before touching memory.
