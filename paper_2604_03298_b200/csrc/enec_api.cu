@@ -495,8 +495,10 @@ enec_status enec_decompress_batched(const enec_batch_item* h_items, int n_items,
     batch.blockwise = 0;
     batch.total_blocks = uint32_t(total);
     bool ticketed = false;
-    if (uint32_t(n_items) <= kInlineJobs) {
-        // a short list travels in the launch parameters: no copy, no scratch
+    // A short list travels in the launch parameters: no copy, no scratch. Unless it has so many blocks that the
+    // ticket of the long-list form (which needs a zeroed word, hence the copy) gains more than the copy costs.
+    constexpr uint64_t kTicketWorthBlocks = 8192;
+    if (uint32_t(n_items) <= kInlineJobs && (capturing != cudaStreamCaptureStatusNone || total < kTicketWorthBlocks)) {
         batch.jobs = nullptr;
         batch.prefix = nullptr;
         for (int i = 0; i < n_items; ++i) batch.inline_jobs[i] = jobs[i];
