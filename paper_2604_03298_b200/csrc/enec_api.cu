@@ -50,7 +50,7 @@ struct ScratchArea {
     bool needs_clear = true;  // compressor areas: fresh memory, a wrapped epoch or a launch that failed
 };
 
-enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1, kScratchCompressBatch = 2, kScratchBlockwise = 3 };
+enum ScratchKind { kScratchCompress = 0, kScratchBatch = 1, kScratchCompressBatch = 2, kScratchBlockwise = 3, kScratchDecodeTicket = 4 };
 
 static std::mutex g_scratch_mu;
 static ScratchArea& scratch_area(int dev, cudaStream_t stream, ScratchKind kind) {
@@ -416,6 +416,28 @@ size_t enec_max_compressed_size(enec_dtype dt, size_t count) {
     return size_t(worst);
 }
 
+// The ticket word of a large tensor's decode launch and the number of the launch on it (see enec_decode_kernel,
+// TICKET = 2). The word is cleared once, when its area is allocated; after that every launch finds the number of an
+// earlier launch in it and starts it afresh.
+static enec_status lease_decode_ticket(int dev, cudaStream_t stream, uint8_t** word, uint32_t* number) {
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    ScratchArea& a = scratch_area(dev, stream, kScratchDecodeTicket);
+    const enec_status st = grow(a, 256);
+    if (st != ENEC_OK) return st;
+    if (a.needs_clear || a.epoch == 0xFFFFFFFFu) {
+        if (cudaMemsetAsync(a.ptr, 0, 256, stream) != cudaSuccess) return ENEC_ERR_CUDA;
+        a.needs_clear = false;
+        a.epoch = 0;
+    }
+    *word = a.ptr;
+    *number = ++a.epoch;
+    return ENEC_OK;
+}
+
+// Tensors of at least this many blocks are decoded with their blocks handed out by a ticket (outside a stream
+// capture: the ticket word carries the launch's number, which a replay would repeat).
+constexpr uint32_t kDecodeTicketMinBlocks = 16384;
+
 static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
                                   int* d_status, cudaStream_t stream, bool ranked, bool blockwise = false) {
     if (!known_dtype(dt)) return ENEC_ERR_UNSUPPORTED_DTYPE;
@@ -432,7 +454,22 @@ static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype d
                                      uint64_t(in_size)};
     batch.inline_prefix[0] = 0;
     batch.inline_prefix[1] = batch.total_blocks;
-    return launch_decode_any(dt, batch, d_status, stream, ranked);
+    int ticketed = 0;
+    if (!ranked && !blockwise && batch.total_blocks >= kDecodeTicketMinBlocks) {
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return ENEC_ERR_CUDA;
+        if (capturing == cudaStreamCaptureStatusNone) {
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
+            uint8_t* word = nullptr;
+            uint32_t number = 0;
+            const enec_status st = lease_decode_ticket(dev, stream, &word, &number);
+            if (st != ENEC_OK) return st;
+            batch.inline_jobs[1] = DecodeJob{word, nullptr, uint64_t(number), 0};  // not a tensor: n_jobs stays 1
+            ticketed = 2;
+        }
+    }
+    return launch_decode_any(dt, batch, d_status, stream, ranked, ticketed);
 }
 
 enec_status enec_decompress(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,

@@ -671,6 +671,7 @@ constexpr uint32_t kInlineJobs = 16;  // tensors of a short batch that fit the k
 // device arrays are laid out as [jobs | prefix, padded to 16 bytes | ticket word, 16 bytes, zero at launch | the
 // tensor of every chunk's first block], so the kernel finds the last two behind the prefix.
 constexpr uint32_t kTicketChunk = 8;
+constexpr uint32_t kSingleTicketChunk = 2;  // one large tensor: its blocks all cost the same, and a launch has few per CTA
 __host__ __device__ inline uint64_t ticket_offset_behind_prefix(uint32_t n_jobs) {
     return align16((uint64_t(n_jobs) + 1) * sizeof(uint32_t));
 }
@@ -743,7 +744,11 @@ __device__ __forceinline__ void prefetch_before_wait(const DecodeBatch& batch, u
 // MAPPED: the instance for streams of the frequency-rank variant (general block body with table look-ups only);
 // each instance refuses the other kind of stream. TICKET: blocks are handed out by batch.ticket; the loader ends the
 // consumers' loop with a descriptor of zero length.
-template <int DT, bool MAPPED = false, bool TICKET = false>
+// TICKET = 2: one large tensor. The ticket is a 64-bit word of the library's scratch that is never cleared: its high
+// half is the number of the launch that uses it (inline_jobs[1].count; the word's address is inline_jobs[1].in), and
+// the first CTA to find another number there starts it at zero for this launch (all earlier launches of the stream
+// have ended by then). In both forms CTA c starts on chunk c without asking, and tickets count on from the grid size.
+template <int DT, bool MAPPED = false, int TICKET = 0>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
 enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -756,7 +761,13 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
     const uint32_t first_block = uint32_t(uint64_t(blockIdx.x) * batch.total_blocks / gridDim.x);
     const uint32_t end_block = uint32_t(uint64_t(blockIdx.x + 1) * batch.total_blocks / gridDim.x);
     const uint32_t n_mine = end_block - first_block;
-    if (threadIdx.x == kConsumerWarps * 32) prefetch_before_wait<DT, MAPPED>(batch, first_block, n_mine);
+    if (threadIdx.x == kConsumerWarps * 32) {
+        if constexpr (TICKET == 2)  // the CTA's first chunk
+            prefetch_before_wait<DT, MAPPED>(batch, blockIdx.x * kSingleTicketChunk,
+                                             blockIdx.x * kSingleTicketChunk < batch.total_blocks ? kSingleTicketChunk : 0);
+        else
+            prefetch_before_wait<DT, MAPPED>(batch, first_block, n_mine);
+    }
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < S; ++s) {
             mbar_init(&ctl->full[s], 1);
@@ -795,22 +806,41 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
         // and the blocks of the chunk in hand that are issued
         [[maybe_unused]] uint32_t chunk = 0, next_chunk = 0, in_chunk = 0;
         [[maybe_unused]] uint32_t next_j = 0, next_first = 0, next_end = 0;  // the next chunk's tensor and its range of blocks
-        [[maybe_unused]] const uint32_t n_chunks = TICKET ? (batch.total_blocks + kTicketChunk - 1) / kTicketChunk : 0;
+        constexpr uint32_t kChunk = TICKET == 2 ? kSingleTicketChunk : kTicketChunk;
+        [[maybe_unused]] const uint32_t n_chunks = TICKET ? (batch.total_blocks + kChunk - 1) / kChunk : 0;
         [[maybe_unused]] uint32_t* const ticket =
-            TICKET ? reinterpret_cast<uint32_t*>(reinterpret_cast<uintptr_t>(batch.prefix) + ticket_offset_behind_prefix(batch.n_jobs))
-                   : nullptr;
-        [[maybe_unused]] const uint32_t* const chunk_job = TICKET ? ticket + 4 : nullptr;
+            TICKET == 1 ? reinterpret_cast<uint32_t*>(reinterpret_cast<uintptr_t>(batch.prefix) + ticket_offset_behind_prefix(batch.n_jobs))
+                        : nullptr;
+        [[maybe_unused]] const uint32_t* const chunk_job = TICKET == 1 ? ticket + 4 : nullptr;
+        [[maybe_unused]] unsigned long long* const ticket64 =
+            TICKET == 2 ? reinterpret_cast<unsigned long long*>(const_cast<uint8_t*>(batch.inline_jobs[1].in)) : nullptr;
+        [[maybe_unused]] auto take_ticket = [&]() -> uint32_t {
+            if constexpr (TICKET == 2) return gridDim.x + uint32_t(atomicAdd(ticket64, 1ull));
+            else return gridDim.x + atomicAdd(ticket, 1u);
+        };
         [[maybe_unused]] auto look_up_next = [&]() {
-            if (next_chunk < n_chunks) {
-                next_j = chunk_job[next_chunk];
-                next_first = prefix[next_j];
-                next_end = prefix[next_j + 1];
+            if constexpr (TICKET == 1) {
+                if (next_chunk < n_chunks) {
+                    next_j = chunk_job[next_chunk];
+                    next_first = prefix[next_j];
+                    next_end = prefix[next_j + 1];
+                }
+            } else {  // one tensor
+                next_j = 0;
+                next_first = 0;
+                next_end = batch.total_blocks;
             }
         };
         if constexpr (TICKET) {
-            chunk = atomicAdd(ticket, 1u);
-            next_chunk = atomicAdd(ticket, 1u);
-            if (chunk < n_chunks) j = chunk_job[chunk];
+            if constexpr (TICKET == 2) {
+                const unsigned long long mine = (unsigned long long)uint32_t(batch.inline_jobs[1].count) << 32;
+                unsigned long long seen;
+                asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(ticket64) : "memory");
+                if ((seen >> 32) != (mine >> 32)) atomicCAS(ticket64, seen, mine);  // one CTA wins; the others find it done
+            }
+            chunk = blockIdx.x;
+            next_chunk = take_ticket();
+            if constexpr (TICKET == 1) { if (chunk < n_chunks) j = chunk_job[chunk]; }
             look_up_next();
         } else {
             uint32_t lo = 0, hi = batch.n_jobs;  // largest j with prefix[j] <= first_block
@@ -834,19 +864,19 @@ enec_decode_kernel(const __grid_constant__ DecodeBatch batch, int* status) {
             uint32_t gb = first_block + issued;
             [[maybe_unused]] bool jumped = false;  // TICKET: this block does not follow the one issued before it
             if constexpr (TICKET) {
-                if (in_chunk == kTicketChunk) {
+                if (in_chunk == kChunk) {
                     chunk = next_chunk;
                     if (chunk >= n_chunks) break;
                     if (next_j != j) parsed = false;
                     j = next_j;
                     job_first = next_first;
                     job_end = next_end;
-                    next_chunk = atomicAdd(ticket, 1u);
+                    next_chunk = take_ticket();
                     look_up_next();
                     in_chunk = 0;
                     jumped = true;
                 }
-                gb = chunk * kTicketChunk + in_chunk;
+                gb = chunk * kChunk + in_chunk;
                 ++in_chunk;
                 if (chunk >= n_chunks || gb >= batch.total_blocks) break;
             }

@@ -3,7 +3,7 @@
 
 namespace enec {
 
-enec_status launch_decode_fp32(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, bool ticketed) {
+enec_status launch_decode_fp32(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, int ticketed) {
     return launch_decode<ENEC_FP32>(batch, d_status, stream, ranked, ticketed);
 }
 

@@ -4,7 +4,7 @@
 namespace enec {
 
 enec_status launch_decode_any(int dt, const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked,
-                              bool ticketed) {
+                              int ticketed) {
     return dt == ENEC_BF16   ? launch_decode_bf16(batch, d_status, stream, ranked, ticketed)
            : dt == ENEC_FP16 ? launch_decode_fp16(batch, d_status, stream, ranked, ticketed)
                              : launch_decode_fp32(batch, d_status, stream, ranked, ticketed);

@@ -25,7 +25,7 @@ inline DecodeDevice* decode_device(int dev) {
 
 template <int DT>
 inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked = false,
-                                 bool ticketed = false) {
+                                 int ticketed = 0) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
     DecodeDevice* found = decode_device(dev);
@@ -36,7 +36,9 @@ inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaSt
                                  int(kDecodeSmemBytes)) != cudaSuccess ||
             cudaFuncSetAttribute(enec_decode_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(kDecodeSmemBytes)) != cudaSuccess ||
-            cudaFuncSetAttribute(enec_decode_kernel<DT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaFuncSetAttribute(enec_decode_kernel<DT, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(kDecodeSmemBytes)) != cudaSuccess ||
+            cudaFuncSetAttribute(enec_decode_kernel<DT, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(kDecodeSmemBytes)) != cudaSuccess)
             return ENEC_ERR_CUDA;
         info.attr_set[DT] = true;
@@ -46,16 +48,18 @@ inline enec_status launch_decode(const DecodeBatch& batch, int* d_status, cudaSt
     if (grid == 0) grid = 1;
     const cudaError_t err =
         ranked         ? launch_pdl(enec_decode_kernel<DT, true>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status)
-        : ticketed     ? launch_pdl(enec_decode_kernel<DT, false, true>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch,
-                                    d_status)
+        : ticketed == 1 ? launch_pdl(enec_decode_kernel<DT, false, 1>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch,
+                                     d_status)
+        : ticketed == 2 ? launch_pdl(enec_decode_kernel<DT, false, 2>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch,
+                                     d_status)
                        : launch_pdl(enec_decode_kernel<DT, false>, grid, kDecodeThreads, kDecodeSmemBytes, stream, batch, d_status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return err == cudaSuccess ? ENEC_OK : ENEC_ERR_CUDA;
 }
 
 
-enec_status launch_decode_bf16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, bool ticketed);
-enec_status launch_decode_fp16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, bool ticketed);
-enec_status launch_decode_fp32(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, bool ticketed);
+enec_status launch_decode_bf16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, int ticketed);
+enec_status launch_decode_fp16(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, int ticketed);
+enec_status launch_decode_fp32(const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked, int ticketed);
 
 }  // namespace enec

@@ -14,9 +14,10 @@ constexpr int kMaxDevices = 64;  // device ordinals the per-device tables cover;
 
 struct DecodeBatch;
 // Launches the decode kernel instance for dt (and for the frequency-rank variant when ranked) over `batch`.
-// ticketed: the batch's device arrays carry a ticket word and the chunk table (see DecodeBatch).
+// ticketed: 1 = the batch's device arrays carry a ticket word and the chunk table, 2 = one tensor with a ticket word
+// of the library's scratch (see DecodeBatch and enec_decode_kernel), 0 = fixed shares of the blocks.
 enec_status launch_decode_any(int dt, const DecodeBatch& batch, int* d_status, cudaStream_t stream, bool ranked,
-                              bool ticketed = false);
+                              int ticketed = 0);
 
 // Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
 // stream drains; it waits for the predecessor's completion itself (pdl_wait) before touching memory.
