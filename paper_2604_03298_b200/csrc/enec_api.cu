@@ -112,8 +112,8 @@ static void place_job(EncodeJob& job, uint8_t* scratch, uint32_t epoch) {
 
 // Tensors of split_min_blocks() .. split_max_blocks() - 1 blocks are compressed in the split form (pack kernel, then
 // the kernel that places the records). Below that range the third launch costs more than the look-back it replaces;
-// above it every CTA has so many blocks that the look-back no longer shows. ENEC_SPLIT_MIN_BLOCKS and
-// ENEC_SPLIT_MAX_BLOCKS in the environment override the bounds (read once; for measurements and tests).
+// there is no upper bound by default. ENEC_SPLIT_MIN_BLOCKS and ENEC_SPLIT_MAX_BLOCKS in the environment override
+// the bounds (read once; for measurements and tests).
 static uint32_t env_blocks(const char* name, uint32_t fallback) {
     const char* e = getenv(name);
     return e && *e ? uint32_t(strtoul(e, nullptr, 10)) : fallback;
@@ -123,7 +123,7 @@ static uint32_t split_min_blocks() {
     return value;
 }
 static uint32_t split_max_blocks() {
-    static const uint32_t value = env_blocks("ENEC_SPLIT_MAX_BLOCKS", 24576u);
+    static const uint32_t value = env_blocks("ENEC_SPLIT_MAX_BLOCKS", 0xFFFFFFFFu);
     return value;
 }
 

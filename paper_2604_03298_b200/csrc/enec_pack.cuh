@@ -262,7 +262,13 @@ enec_pack_tensor_kernel(const EncodeJob job, int* status) {
     const uint32_t slot = record_slot_bytes(n - m);
     const uint8_t* in_base = reinterpret_cast<const uint8_t*>(job.in);
     const uint8_t* in_end = in_base + job.count * kElemBytes;
-    for (uint32_t k = blockIdx.x; k < g.nblocks; k += gridDim.x) {
+    // CTA c takes blocks c and c + grid; after that blocks are handed out by the call's ticket, asked for two blocks
+    // ahead (the CTAs of an SM do not progress equally), so that the answer and the block's L2 prefetch are never waited for
+    __shared__ uint32_t s_next;
+    uint32_t k = blockIdx.x, k_next = blockIdx.x + gridDim.x;
+    for (; k < g.nblocks; ) {
+        uint32_t asked = 0;
+        if (tid == 0) asked = atomicAdd(&job.ctl->ticket, 1u);
         const bool last = k + 1 == g.nblocks;
         const uint32_t N = last ? g.tail_padded : kBlockElems;
         const uint32_t real = last ? g.tail_real : kBlockElems;
@@ -273,8 +279,8 @@ enec_pack_tensor_kernel(const EncodeJob job, int* status) {
         uint8_t* out_smhi = job.out + sec.smhi + uint64_t(k) * (kBlockElems / 8) * 3;
         uint8_t* out_mask = job.out + sec.mask + uint64_t(k) * (kGroupsPerBlock / 8);
         uint8_t* out_rec = job.out + sec.high + uint64_t(k) * slot;
-        {   // the CTA's next block towards L2 (one 128-byte line per thread, two for fp32)
-            const uint8_t* next = in_bytes + uint64_t(gridDim.x) * kBlockElems * kElemBytes;
+        if (k_next < g.nblocks) {   // the CTA's next block towards L2 (one 128-byte line per thread, two for fp32)
+            const uint8_t* next = in_base + uint64_t(k_next) * kBlockElems * kElemBytes;
 #pragma unroll
             for (uint32_t r = 0; r < kElemBytes / 2; ++r) {
                 const uint8_t* line = next + (r * kPackThreads + tid) * 128;
@@ -286,7 +292,14 @@ enec_pack_tensor_kernel(const EncodeJob job, int* status) {
             wide = pack_tail_block<DT>(in_bytes, N, real, b, n, m, out_sm, out_low, out_smhi, out_mask, out_smlo, out_rec, pack_smem);
         else
             wide = pack_full_block<DT>(in_bytes, b, n, m, out_sm, out_smlo, out_low, out_smhi, out_mask, out_rec, pack_smem, s_mask);
-        if (tid == 0) job.state[k] = wide;  // read by the next kernel
+        if (tid == 0) {
+            job.state[k] = wide;  // read by the next kernel
+            s_next = 2 * gridDim.x + asked;
+        }
+        __syncthreads();
+        k = k_next;
+        k_next = s_next;
+        __syncthreads();  // s_next is read before the next round's write
     }
     (void)status;
 }
