@@ -27,7 +27,8 @@
  * enec_compress / enec_compress_with_params / enec_compress_batched on a stream that is being captured into a
  * CUDA graph return ENEC_ERR_INVALID_ARG (a replay would not see the state). Decompression can be captured: what
  * it keeps per (device, stream) is one word that hands out the blocks of tensors of about 2^28 elements or more (allocated
- * with the first such call on the stream, numbered per launch, never relied on by a later call), and a call on a
+ * with the first such call on the stream, numbered per launch, never relied on by a later call; if it cannot be
+ * allocated the call does without it), and a call on a
  * capturing stream does without it; a batched call of more than 16 tensors is then recorded as one launch per 16 tensors, since
  * a longer list would have to pass through host and scratch memory that a replay cannot rely on.
  */

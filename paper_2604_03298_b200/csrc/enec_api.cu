@@ -463,10 +463,11 @@ static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype d
             if (cudaGetDevice(&dev) != cudaSuccess) return ENEC_ERR_CUDA;
             uint8_t* word = nullptr;
             uint32_t number = 0;
-            const enec_status st = lease_decode_ticket(dev, stream, &word, &number);
-            if (st != ENEC_OK) return st;
-            batch.inline_jobs[1] = DecodeJob{word, nullptr, uint64_t(number), 0};  // not a tensor: n_jobs stays 1
-            ticketed = 2;
+            // without the word (no device memory to be had) the launch keeps fixed shares: slower, not wrong
+            if (lease_decode_ticket(dev, stream, &word, &number) == ENEC_OK) {
+                batch.inline_jobs[1] = DecodeJob{word, nullptr, uint64_t(number), 0};  // not a tensor: n_jobs stays 1
+                ticketed = 2;
+            }
         }
     }
     return launch_decode_any(dt, batch, d_status, stream, ranked, ticketed);
