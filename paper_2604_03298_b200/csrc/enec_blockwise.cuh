@@ -45,7 +45,8 @@ struct BlockwiseJob {
     const uint16_t* in;
     uint8_t* out;
     uint64_t count;
-    uint32_t* done;                // blocks whose entry is written (zero when the call starts)
+    uint32_t* done;                // blocks whose entry is written (zero when the call starts); done[1] and done[2] are
+                                   // the tickets that hand out the blocks in the two kernels (each zeroed by the other kernel)
     unsigned long long* out_size;  // device, may be null
 };
 
@@ -176,7 +177,13 @@ enec_block_params_kernel(const BlockwiseJob job, int* status) {
     pdl_wait();  // nothing above touches global memory
     const Geometry g = make_geometry(job.count);
     BlockEntry* table = reinterpret_cast<BlockEntry*>(job.out + kHeaderBytes);
-    for (uint32_t k = blockIdx.x; k < g.nblocks; k += gridDim.x) {
+    // CTA c starts on block c; after that blocks are handed out by a ticket, asked for a block ahead (the CTAs of an
+    // SM do not progress equally). The pack kernel's ticket, last used by the call before, is cleared here.
+    __shared__ uint32_t s_next_block;
+    if (blockIdx.x == 0 && tid == 0) job.done[2] = 0;
+    for (uint32_t k = blockIdx.x; k < g.nblocks;) {
+        uint32_t asked = 0;
+        if (tid == 0) asked = atomicAdd(&job.done[1], 1u);
         const bool last = k + 1 == g.nblocks;
         const uint32_t N = last ? g.tail_padded : kBlockElems;
         const uint32_t real = last ? g.tail_real : kBlockElems;
@@ -239,8 +246,10 @@ enec_block_params_kernel(const BlockwiseJob job, int* status) {
             table[k] = e;
             __threadfence();
             s_last = atomicAdd(job.done, 1u) + 1 == g.nblocks;
+            s_next_block = gridDim.x + asked;
         }
         __syncthreads();
+        k = s_next_block;
         if (s_last) {
             __threadfence();
             finish_block_table<DT>(job, g);
@@ -264,7 +273,15 @@ enec_pack_blocks_kernel(const BlockwiseJob job, int* status) {
     const uint32_t m_tail = table[g.nblocks - 1].m;
     const uint64_t low_bytes = uint64_t(totals.m_before - m_tail) * (kBlockElems / 8) + uint64_t(g.tail_padded) * m_tail / 8;
     const Sections sec = make_sections_blockwise(DT, job.count, g, low_bytes, totals.rec_before);
-    for (uint32_t k = blockIdx.x; k < g.nblocks; k += gridDim.x) {
+    // blocks c and c + grid, then blocks handed out by the call's second ticket, asked for two blocks ahead; the first
+    // kernel's ticket is cleared here for the next call
+    __shared__ uint32_t s_next;
+    const uint32_t tid = threadIdx.x;
+    if (blockIdx.x == 0 && tid == 0) job.done[1] = 0;
+    uint32_t k = blockIdx.x, k_next = blockIdx.x + gridDim.x;
+    while (k < g.nblocks) {
+        uint32_t asked = 0;
+        if (tid == 0) asked = atomicAdd(&job.done[2], 1u);
         const BlockEntry entry = table[k];
         const int b = entry.b, n = entry.n, m = entry.m;
         const bool last = k + 1 == g.nblocks;
@@ -281,6 +298,11 @@ enec_pack_blocks_kernel(const BlockwiseJob job, int* status) {
             pack_tail_block<DT>(in_bytes, N, real, b, n, m, out_sm, out_low, out_smhi, out_mask, out_smlo, out_rec, pack_smem);
         else
             pack_full_block<DT>(in_bytes, b, n, m, out_sm, out_smlo, out_low, out_smhi, out_mask, out_rec, pack_smem, s_mask);
+        if (tid == 0) s_next = 2 * gridDim.x + asked;
+        __syncthreads();
+        k = k_next;
+        k_next = s_next;
+        __syncthreads();  // s_next is read before the next round's write
     }
     (void)status;
 }
