@@ -213,8 +213,9 @@ static enec_status launch_encode_batched(const EncodeJob* d_jobs, const HistUnit
     }
     uint32_t grid = uint32_t(info.sms) * 3;
     if (grid > n_units) grid = n_units;
-    if (launch_pdl(enec_histogram_batched_kernel<DT>, grid, kHistThreads, hist_smem, stream, d_jobs, d_units, n_units) !=
-        cudaSuccess)
+    // the second word of the call's ticket area hands out the histogram units (the first one the blocks of the encode)
+    if (launch_pdl(enec_histogram_batched_kernel<DT>, grid, kHistThreads, hist_smem, stream, d_jobs, d_units, n_units,
+                   batch.ticket + 4) != cudaSuccess)
         return ENEC_ERR_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     grid = uint32_t(info.sms) * 4;

@@ -380,7 +380,8 @@ struct HistUnit {
 
 template <int DT>
 __global__ void __launch_bounds__(kHistThreads, 3)
-enec_histogram_batched_kernel(const EncodeJob* __restrict__ jobs, const HistUnit* __restrict__ units, uint32_t n_units) {
+enec_histogram_batched_kernel(const EncodeJob* __restrict__ jobs, const HistUnit* __restrict__ units, uint32_t n_units,
+                              uint32_t* ticket) {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t cta_hist[256];
     __shared__ int s_last;
@@ -393,7 +394,12 @@ enec_histogram_batched_kernel(const EncodeJob* __restrict__ jobs, const HistUnit
     cta_hist[tid] = 0;
     __syncthreads();
     pdl_wait();  // nothing above touches global memory
-    for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
+    // CTA c starts on unit c; after that units are handed out by `ticket` (zero when the launch starts), asked for
+    // a unit ahead: the CTAs of an SM do not progress equally
+    __shared__ uint32_t s_next_unit;
+    for (uint32_t u = blockIdx.x; u < n_units;) {
+        uint32_t asked = 0;
+        if (tid == 0) asked = atomicAdd(ticket, 1u);
         const HistUnit unit = units[u];
         const uint16_t* in = jobs[unit.job].in;
         const uint64_t count = jobs[unit.job].count;
@@ -436,8 +442,12 @@ enec_histogram_batched_kernel(const EncodeJob* __restrict__ jobs, const HistUnit
         cta_hist[tid] = 0;
         __threadfence();
         __syncthreads();
-        if (tid == 0) s_last = atomicAdd(&ctl->hist_done, 1u) == unit.units_of_job - 1;
+        if (tid == 0) {
+            s_last = atomicAdd(&ctl->hist_done, 1u) == unit.units_of_job - 1;
+            s_next_unit = gridDim.x + asked;
+        }
         __syncthreads();
+        u = s_next_unit;
         if (s_last) {
             __threadfence();
             parameter_search<DT>(ctl);
