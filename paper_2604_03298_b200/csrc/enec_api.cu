@@ -436,8 +436,12 @@ static enec_status lease_decode_ticket(int dev, cudaStream_t stream, uint8_t** w
 }
 
 // Tensors of at least this many blocks are decoded with their blocks handed out by a ticket (outside a stream
-// capture: the ticket word carries the launch's number, which a replay would repeat).
-constexpr uint32_t kDecodeTicketMinBlocks = 16384;
+// capture: the ticket word carries the launch's number, which a replay would repeat). ENEC_DECODE_TICKET_MIN_BLOCKS
+// in the environment overrides the bound (read once; for measurements and tests).
+static uint32_t decode_ticket_min_blocks() {
+    static const uint32_t value = env_blocks("ENEC_DECODE_TICKET_MIN_BLOCKS", 16384u);
+    return value;
+}
 
 static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype dt, size_t count, void* d_out,
                                   int* d_status, cudaStream_t stream, bool ranked, bool blockwise = false) {
@@ -456,7 +460,7 @@ static enec_status decompress_one(const void* d_in, size_t in_size, enec_dtype d
     batch.inline_prefix[0] = 0;
     batch.inline_prefix[1] = batch.total_blocks;
     int ticketed = 0;
-    if (!ranked && !blockwise && batch.total_blocks >= kDecodeTicketMinBlocks) {
+    if (!ranked && !blockwise && batch.total_blocks >= decode_ticket_min_blocks()) {
         cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
         if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return ENEC_ERR_CUDA;
         if (capturing == cudaStreamCaptureStatusNone) {

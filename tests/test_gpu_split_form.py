@@ -1,7 +1,8 @@
-"""GPU parity for the two-kernel form of enec_compress (pack kernel + the kernel that moves every block's records to
-their offsets, Sec. 5.1 / 5.4). The library takes that form for tensors of some thousand blocks; here a child process
-lowers the bound through the environment so that small tensors, tails and all dtypes go through it too, and compares
-every stream with the oracle's byte for byte. (The bound is read once per process, hence the child.)"""
+"""GPU parity for two forms the library takes only for large tensors: the two-kernel form of enec_compress (pack kernel
++ the kernel that moves every block's records to their offsets, Sec. 5.1 / 5.4) and the decoder that hands a tensor's
+blocks out by a ticket. Here a child process lowers their bounds through the environment so that small tensors, tails
+and all dtypes go through them too, and compares every stream with the oracle's byte for byte and every decoded
+tensor bit for bit. (The bounds are read once per process, hence the child.)"""
 import os
 import subprocess
 import sys
@@ -76,7 +77,7 @@ print("split form ok", len(launches_per_call))
 
 
 def test_split_form_writes_the_oracles_streams():
-    env = dict(os.environ, ENEC_SPLIT_MIN_BLOCKS="1", ENEC_SPLIT_MAX_BLOCKS="100000000")
+    env = dict(os.environ, ENEC_SPLIT_MIN_BLOCKS="1", ENEC_SPLIT_MAX_BLOCKS="100000000", ENEC_DECODE_TICKET_MIN_BLOCKS="1")
     res = subprocess.run([sys.executable, "-c", "ROOT = %r\n" % ROOT + CHILD], env=env, capture_output=True, text=True,
                          timeout=900)
     assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-4000:]
